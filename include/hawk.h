@@ -1,0 +1,158 @@
+/*
+ * hawk.h - C ABI of the B200 (sm_100a) verify step of speculative decoding for autoregressive
+ * image generation (Hawk).
+ *
+ * The verify step takes a block of K drafted image tokens per sequence and decides how many of
+ * them the target model accepts.  It has three parts, one entry point each:
+ *   hawk_verify_attn  block-causal attention of the K draft queries over the cached context, for
+ *                     the conditional and the unconditional guidance stream;
+ *   hawk_head_proj    projection of the K hidden states onto the image-token codebook;
+ *   hawk_cfg_accept   guidance combine, temperature, top-k, softmax and speculative rejection
+ *                     sampling, returning the accepted length and the correction token.
+ *
+ * Conventions common to all entry points
+ *   - Every pointer is a DEVICE pointer owned by the caller unless the comment says "host".  The
+ *     library allocates nothing, frees nothing, never synchronises and keeps no pointer after
+ *     the call returns.  All work is queued on `stream`.
+ *   - Tensors are dense, row-major in the index order written in brackets, base address aligned
+ *     to 16 bytes.  bf16 is the 16 high bits of an IEEE fp32.
+ *   - The return value is the only error channel.  On any error nothing is launched and the
+ *     outputs are untouched.  Conditions that only the device can see (a draft id out of range,
+ *     a NaN logit, a wait that ran out) are OR-ed into *dev_status (HAWK_DEV_* bits) when that
+ *     pointer is not NULL; the caller clears the word.  No kernel traps or asserts.
+ *   - B sequences, S = 2B guidance streams: stream b is the conditional one of sequence b,
+ *     stream B+b its unconditional one.  K drafts per sequence.
+ */
+#ifndef HAWK_H
+#define HAWK_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct CUstream_st *hawk_stream_t; /* a cudaStream_t / CUstream; 0 = the default stream */
+
+typedef enum {
+    HAWK_OK = 0,
+    HAWK_ERR_NULL = 1,        /* a required pointer is NULL                                     */
+    HAWK_ERR_SHAPE = 2,       /* a size is negative or sizes contradict each other              */
+    HAWK_ERR_ALIGN = 3,       /* a tensor base is not 16-byte aligned                           */
+    HAWK_ERR_UNSUPPORTED = 4, /* a value outside what the kernels are built for (see each call) */
+    HAWK_ERR_WORKSPACE = 5,   /* workspace missing or smaller than *_workspace_bytes says       */
+    HAWK_ERR_PARAM = 6,       /* a scalar parameter is not a usable number                      */
+    HAWK_ERR_CUDA = 7         /* the CUDA runtime or driver refused a call (launch, tensor map) */
+} hawk_status;
+
+/* bits of *dev_status */
+#define HAWK_DEV_TIMEOUT 1    /* a bounded wait inside a kernel ran out; outputs are not valid  */
+#define HAWK_DEV_BAD_DRAFT 2  /* a draft id lay outside [v_begin, v_end) and was clamped into it */
+#define HAWK_DEV_NONFINITE 4  /* a NaN or +inf logit was treated as -inf                        */
+#define HAWK_DEV_BAD_PREFIX 8 /* a prefix length lay outside [0, L_cap - K] and was clamped     */
+
+const char *hawk_status_string(hawk_status status);
+int hawk_version(void); /* major*10000 + minor*100 + patch */
+
+/* ------------------------------------------------------------------------------------------------
+ * hawk_verify_attn - attention of the K draft queries against the cached prefix.
+ *
+ * Operation (Sec. 3, "Speculative Sampling": one forward pass of the target model verifies the
+ * drafted tokens in parallel; the KV cache is the one App. C mentions).  For stream s, query head
+ * h and draft position i, with n = prefix_len[s] + i + 1 visible keys and kv head g = h / (H/H_kv):
+ *     e_j = sm_scale * <q[s,i,h,:], k_cache[s,g,j,:]>,  j < n
+ *     out[s,i,h*D:(h+1)*D] = sum_j softmax(e)_j * v_cache[s,g,j,:]
+ * The block's own K rows must already be stored in the caches at rows prefix_len[s] .. +K-1; rows
+ * past that are never used (they may hold anything).  Scores and sums are fp32.
+ *
+ *   q            bf16 [S][K][H][D]
+ *   k_cache      bf16 [S][H_kv][L_cap][D]
+ *   v_cache      bf16 [S][H_kv][L_cap][D]
+ *   prefix_len   int32 [S], each in [0, L_cap - K]
+ *   out          bf16 [S][K][H*D]
+ *   max_prefix_len  upper bound of prefix_len[] known on the host (sizes the launch only)
+ *   sm_scale     score scale, > 0, normally 1/sqrt(D)
+ *   workspace    scratch of at least hawk_verify_attn_workspace_bytes(...) bytes, 16-byte aligned;
+ *                may be NULL when that function returns 0.  Contents need no initialisation and
+ *                are garbage afterwards.
+ * Supported: D in {64, 128}; 1 <= K <= 16; H a multiple of H_kv; S*H_kv*L_cap < 2^31.
+ * Errors: NULL, SHAPE (negative sizes, max_prefix_len + K > L_cap), ALIGN, UNSUPPORTED, WORKSPACE,
+ * PARAM (sm_scale not a positive finite number), CUDA.  S == 0 returns HAWK_OK without a launch.
+ * ---------------------------------------------------------------------------------------------- */
+size_t hawk_verify_attn_workspace_bytes(int S, int K, int H, int H_kv, int D, int max_prefix_len);
+
+hawk_status hawk_verify_attn(const void *q, const void *k_cache, const void *v_cache,
+                             const int32_t *prefix_len, void *out, int S, int K, int H, int H_kv,
+                             int D, int L_cap, int max_prefix_len, float sm_scale, void *workspace,
+                             size_t workspace_bytes, int32_t *dev_status, hawk_stream_t stream);
+
+/* ------------------------------------------------------------------------------------------------
+ * hawk_head_proj - output head: hidden states onto the token codebook.
+ *
+ * Operation (Sec. 3: the decoding head after the final hidden layer maps a hidden state to
+ * logits over the codebook of image tokens):
+ *     logits[m][v] = sum_c x[m][c] * w[v][c]      for v_begin <= v < v_end
+ * bf16 operands, fp32 accumulation on the tensor cores, fp32 result.  Columns outside
+ * [v_begin, v_end) are not written.
+ *
+ *   x       bf16 [M][hidden]   one row per (stream, draft position): M = 2*B*K
+ *   w       bf16 [V][hidden]   one row per token id
+ *   logits  fp32 [M][V]
+ * Supported: hidden a multiple of 64; V a multiple of 4 and logits 16-byte aligned.
+ * Errors: NULL, SHAPE (negative sizes, range outside [0, V]), ALIGN, UNSUPPORTED, CUDA.
+ * M == 0 or an empty range returns HAWK_OK without a launch.
+ * ---------------------------------------------------------------------------------------------- */
+hawk_status hawk_head_proj(const void *x, const void *w, float *logits, int M, int hidden, int V,
+                           int v_begin, int v_end, int32_t *dev_status, hawk_stream_t stream);
+
+/* ------------------------------------------------------------------------------------------------
+ * hawk_cfg_accept - target distribution and speculative rejection sampling of a draft chain.
+ *
+ * Operation, per sequence b and draft position i = 0, 1, ... (Sec. 3: accept draft x with
+ * probability min(1, p(x)/q(x)), otherwise resample from norm(max(0, p - q)); Sec. 4.2, Eq.
+ * "recur": a pass moves one position deeper, the first rejection ends the chain; generation
+ * settings of Sec. 5: guidance scale, temperature, top-k):
+ *   1. l[v] = lu[v] + cfg_scale*(lc[v] - lu[v]) over the valid ids, lc/lu the conditional and
+ *      unconditional logit rows; -inf in either gives -inf.  Evaluated in fp32 as subtract, fused
+ *      multiply-add, then divide by temperature.
+ *   2. With 0 < top_k < number of finite l: keep every l >= the top_k-th largest (ties at the
+ *      threshold are all kept); the rest become -inf.
+ *   3. p = softmax(l); ids outside [v_begin, v_end) have p = 0.
+ *   4. x = draft[b][i]; accept iff u_accept[b][i] * q[b][i][x] < p[x]; on a pass go to i+1.
+ *   5. On the first rejection: r = max(0, p - q[b][i][:]); if r has no mass, r = p;
+ *      out_token[b] = the smallest id whose running sum of r (ascending id) exceeds
+ *      u_resample[b][i] * sum(r); accept_len[b] = i.
+ *   6. All K accepted: accept_len[b] = K; out_token[b] = -1, or with has_bonus_row the same draw
+ *      from p of row K with u_resample[b][K].
+ * The paper's "accept length" counts the correction token: it equals accept_len + 1.
+ *
+ *   logits      fp32 [2B][K + has_bonus_row][V]
+ *   q_probs     fp32 [B][K][V]   draft probabilities, used as given
+ *   draft       int32 [B][K]
+ *   u_accept    fp32 [B][K]      uniforms in [0,1)
+ *   u_resample  fp32 [B][K+1]    uniforms in [0,1)
+ *   accept_len  int32 [B]  (out)
+ *   out_token   int32 [B]  (out)
+ *   p_debug     optional fp32 [B][K + has_bonus_row][V]: receives p over the valid ids; NULL in
+ *               normal use (p never leaves the chip)
+ *   workspace   at least hawk_cfg_accept_workspace_bytes(...) bytes, 16-byte aligned; needs no
+ *               initialisation
+ * Supported: 1 <= K <= 16; 1 <= v_end - v_begin <= 32768 (one row is held in one
+ * thread block's registers); temperature > 0.
+ * Errors: NULL, SHAPE, ALIGN, UNSUPPORTED, WORKSPACE, PARAM (cfg_scale or temperature not finite,
+ * temperature <= 0), CUDA.  B == 0 returns HAWK_OK without a launch.
+ * ---------------------------------------------------------------------------------------------- */
+size_t hawk_cfg_accept_workspace_bytes(int B, int K, int V);
+
+hawk_status hawk_cfg_accept(const float *logits, const float *q_probs, const int32_t *draft,
+                            const float *u_accept, const float *u_resample, int B, int K, int V,
+                            int v_begin, int v_end, float cfg_scale, float temperature, int top_k,
+                            int has_bonus_row, int32_t *accept_len, int32_t *out_token,
+                            float *p_debug, void *workspace, size_t workspace_bytes,
+                            int32_t *dev_status, hawk_stream_t stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* HAWK_H */

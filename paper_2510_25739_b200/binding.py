@@ -1,0 +1,182 @@
+"""Thin Python binding of the C-ABI library: argument marshalling only.
+
+Every function takes torch CUDA tensors, checks dtype/contiguity/device, and passes raw pointers,
+sizes and the current CUDA stream to the entry point of the same name in libhawk_verify.so.  No
+step of the verify path is computed here, and there is no fallback: a missing library raises.
+"""
+from __future__ import annotations
+
+import ctypes
+from pathlib import Path
+from typing import Optional
+
+import torch
+
+_PKG = Path(__file__).resolve().parent
+_LIB_PATH = _PKG / "libhawk_verify.so"
+_lib: Optional[ctypes.CDLL] = None
+
+DEV_TIMEOUT, DEV_BAD_DRAFT, DEV_NONFINITE, DEV_BAD_PREFIX = 1, 2, 4, 8
+
+EXPORTS = (
+    "hawk_status_string", "hawk_version",
+    "hawk_verify_attn_workspace_bytes", "hawk_verify_attn",
+    "hawk_head_proj",
+    "hawk_cfg_accept_workspace_bytes", "hawk_cfg_accept",
+)
+
+
+class HawkError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        super().__init__(f"{where}: status {code} ({status_string(code)})")
+
+
+def library_path() -> Path:
+    return _LIB_PATH
+
+
+def load_library() -> ctypes.CDLL:
+    """Loads libhawk_verify.so (built in-tree by paper_2510_25739_b200.build); raises if absent."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not _LIB_PATH.exists():
+        raise RuntimeError(
+            f"{_LIB_PATH} is missing: build it with `python -m paper_2510_25739_b200.build` "
+            "(or __graft_entry__.build()); there is no fallback path")
+    lib = ctypes.CDLL(str(_LIB_PATH))
+    vp, i32, f32, sz = ctypes.c_void_p, ctypes.c_int, ctypes.c_float, ctypes.c_size_t
+    lib.hawk_status_string.restype = ctypes.c_char_p
+    lib.hawk_status_string.argtypes = [i32]
+    lib.hawk_version.restype = i32
+    lib.hawk_version.argtypes = []
+    lib.hawk_verify_attn_workspace_bytes.restype = sz
+    lib.hawk_verify_attn_workspace_bytes.argtypes = [i32] * 6
+    lib.hawk_verify_attn.restype = i32
+    lib.hawk_verify_attn.argtypes = [vp, vp, vp, vp, vp, i32, i32, i32, i32, i32, i32, i32, f32, vp, sz, vp, vp]
+    lib.hawk_head_proj.restype = i32
+    lib.hawk_head_proj.argtypes = [vp, vp, vp, i32, i32, i32, i32, i32, vp, vp]
+    lib.hawk_cfg_accept_workspace_bytes.restype = sz
+    lib.hawk_cfg_accept_workspace_bytes.argtypes = [i32] * 3
+    lib.hawk_cfg_accept.restype = i32
+    lib.hawk_cfg_accept.argtypes = [vp, vp, vp, vp, vp, i32, i32, i32, i32, i32, f32, f32, i32, i32,
+                                    vp, vp, vp, vp, sz, vp, vp]
+    _lib = lib
+    return lib
+
+
+def status_string(code: int) -> str:
+    return load_library().hawk_status_string(int(code)).decode()
+
+
+def version() -> int:
+    return load_library().hawk_version()
+
+
+def _ptr(t: Optional[torch.Tensor]):
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def _check(t: torch.Tensor, dtype, name: str, shape=None):
+    if t.dtype != dtype:
+        raise TypeError(f"{name}: expected {dtype}, got {t.dtype}")
+    if not t.is_cuda:
+        raise ValueError(f"{name}: must be a CUDA tensor")
+    if not t.is_contiguous():
+        raise ValueError(f"{name}: must be contiguous")
+    if shape is not None and tuple(t.shape) != tuple(shape):
+        raise ValueError(f"{name}: expected shape {tuple(shape)}, got {tuple(t.shape)}")
+
+
+def _stream() -> ctypes.c_void_p:
+    return ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def verify_attn_workspace_bytes(S: int, K: int, H: int, H_kv: int, D: int, max_prefix_len: int) -> int:
+    return int(load_library().hawk_verify_attn_workspace_bytes(S, K, H, H_kv, D, max_prefix_len))
+
+
+def verify_attn(q: torch.Tensor, k_cache: torch.Tensor, v_cache: torch.Tensor, prefix_len: torch.Tensor,
+                max_prefix_len: int, sm_scale: float, out: Optional[torch.Tensor] = None,
+                workspace: Optional[torch.Tensor] = None, dev_status: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """q [S,K,H,D], caches [S,H_kv,L_cap,D] (bf16), prefix_len [S] int32 -> out [S,K,H*D] bf16."""
+    lib = load_library()
+    S, K, H, D = q.shape
+    _, H_kv, L_cap, _ = k_cache.shape
+    _check(q, torch.bfloat16, "q")
+    _check(k_cache, torch.bfloat16, "k_cache", (S, H_kv, L_cap, D))
+    _check(v_cache, torch.bfloat16, "v_cache", (S, H_kv, L_cap, D))
+    _check(prefix_len, torch.int32, "prefix_len", (S,))
+    if out is None:
+        out = torch.empty((S, K, H * D), dtype=torch.bfloat16, device=q.device)
+    _check(out, torch.bfloat16, "out", (S, K, H * D))
+    need = verify_attn_workspace_bytes(S, K, H, H_kv, D, max_prefix_len)
+    if workspace is None and need:
+        workspace = torch.empty(need, dtype=torch.uint8, device=q.device)
+    ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    rc = lib.hawk_verify_attn(_ptr(q), _ptr(k_cache), _ptr(v_cache), _ptr(prefix_len), _ptr(out), S, K, H, H_kv, D,
+                              L_cap, int(max_prefix_len), float(sm_scale), _ptr(workspace), ws_bytes,
+                              _ptr(dev_status), _stream())
+    if rc != 0:
+        raise HawkError(rc, "hawk_verify_attn")
+    return out
+
+
+def head_proj(x: torch.Tensor, w: torch.Tensor, v_begin: int = 0, v_end: Optional[int] = None,
+              logits: Optional[torch.Tensor] = None, dev_status: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """x [M,hidden], w [V,hidden] (bf16) -> logits [M,V] fp32 (only columns [v_begin,v_end) written)."""
+    lib = load_library()
+    M, hidden = x.shape
+    V = w.shape[0]
+    v_end = V if v_end is None else v_end
+    _check(x, torch.bfloat16, "x")
+    _check(w, torch.bfloat16, "w", (V, hidden))
+    if logits is None:
+        logits = torch.empty((M, V), dtype=torch.float32, device=x.device)
+    _check(logits, torch.float32, "logits", (M, V))
+    rc = lib.hawk_head_proj(_ptr(x), _ptr(w), _ptr(logits), M, hidden, V, int(v_begin), int(v_end),
+                            _ptr(dev_status), _stream())
+    if rc != 0:
+        raise HawkError(rc, "hawk_head_proj")
+    return logits
+
+
+def cfg_accept_workspace_bytes(B: int, K: int, V: int) -> int:
+    return int(load_library().hawk_cfg_accept_workspace_bytes(B, K, V))
+
+
+def cfg_accept(logits: torch.Tensor, q_probs: torch.Tensor, draft: torch.Tensor, u_accept: torch.Tensor,
+               u_resample: torch.Tensor, v_begin: int, v_end: int, cfg_scale: float, temperature: float,
+               top_k: int, has_bonus_row: bool = False, accept_len: Optional[torch.Tensor] = None,
+               out_token: Optional[torch.Tensor] = None, p_debug: Optional[torch.Tensor] = None,
+               workspace: Optional[torch.Tensor] = None, dev_status: Optional[torch.Tensor] = None):
+    """logits [2B,K(+1),V] fp32, q_probs [B,K,V] fp32, draft [B,K] int32, uniforms -> (accept_len, out_token)."""
+    lib = load_library()
+    B, K, V = q_probs.shape
+    rows = K + (1 if has_bonus_row else 0)
+    _check(logits, torch.float32, "logits", (2 * B, rows, V))
+    _check(q_probs, torch.float32, "q_probs")
+    _check(draft, torch.int32, "draft", (B, K))
+    _check(u_accept, torch.float32, "u_accept", (B, K))
+    _check(u_resample, torch.float32, "u_resample", (B, K + 1))
+    dev = logits.device
+    if accept_len is None:
+        accept_len = torch.empty(B, dtype=torch.int32, device=dev)
+    if out_token is None:
+        out_token = torch.empty(B, dtype=torch.int32, device=dev)
+    _check(accept_len, torch.int32, "accept_len", (B,))
+    _check(out_token, torch.int32, "out_token", (B,))
+    if p_debug is not None:
+        _check(p_debug, torch.float32, "p_debug", (B, rows, V))
+    need = cfg_accept_workspace_bytes(B, K, V)
+    if workspace is None:
+        workspace = torch.empty(max(need, 16), dtype=torch.uint8, device=dev)
+    ws_bytes = workspace.numel() * workspace.element_size()
+    rc = lib.hawk_cfg_accept(_ptr(logits), _ptr(q_probs), _ptr(draft), _ptr(u_accept), _ptr(u_resample), B, K, V,
+                             int(v_begin), int(v_end), float(cfg_scale), float(temperature), int(top_k),
+                             int(bool(has_bonus_row)), _ptr(accept_len), _ptr(out_token), _ptr(p_debug),
+                             _ptr(workspace), ws_bytes, _ptr(dev_status), _stream())
+    if rc != 0:
+        raise HawkError(rc, "hawk_cfg_accept")
+    return accept_len, out_token

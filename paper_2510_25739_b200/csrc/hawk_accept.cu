@@ -1,0 +1,559 @@
+// hawk_cfg_accept: guidance combine, temperature, top-k, softmax, acceptance test and residual
+// resampling, one thread block per (sequence, draft position) row.
+//
+// The row of guided logits lives in registers from the moment it is read (each logit row is read
+// from HBM exactly once); the target probabilities p and the residual max(0, p - q) are never
+// written back.  Draft probabilities q are read only by rows whose draft was rejected.
+// A second, tiny kernel picks, per sequence, the first rejected row.
+//
+// Rule implemented: accept draft x iff u * q(x) < p(x); at the first rejection draw the
+// correction token from norm(max(0, p - q)) by inverse CDF in ascending token id
+// (speculative sampling, Sec. 3; chain verification and residual update, Sec. 4.2).
+#include <math_constants.h>
+
+#include "hawk_common.cuh"
+
+namespace {
+
+constexpr int kBins = 2048;     // histogram bins of one top-k selection round
+constexpr int kCandMax = 2048;  // candidates ranked exactly in shared memory
+constexpr int kMaxRounds = 48;  // each round shrinks the value range by >= 2048x; fp32 allows < 16
+
+constexpr int ROW_ACCEPTED = -1;
+constexpr int ROW_REJECTED_NO_TOKEN = -2;  // rejected and nothing has positive mass
+
+struct AcceptParams {
+    const float *logits;
+    const float *q;
+    const int32_t *draft;
+    const float *u_acc;
+    const float *u_res;
+    int B, K, rows, V, v_begin, n;
+    float cfg_scale, temperature;
+    int top_k;
+    int vec_ok;
+    int32_t *row_out;  // [B][rows]
+    float *p_debug;
+    int32_t *dev_status;
+};
+
+__device__ __forceinline__ float4 ld_stream4(const float *p)
+{
+    return __ldcs(reinterpret_cast<const float4 *>(p));
+}
+
+// Loads 4 consecutive floats starting at element e of a row of n valid elements; elements past
+// the row end read as `fill`.
+__device__ __forceinline__ float4 load4(const float *row, int e, int n, bool vec_ok, float fill)
+{
+    if (vec_ok && e + 3 < n) return ld_stream4(row + e);
+    float4 r;
+    r.x = e + 0 < n ? __ldcs(row + e + 0) : fill;
+    r.y = e + 1 < n ? __ldcs(row + e + 1) : fill;
+    r.z = e + 2 < n ? __ldcs(row + e + 2) : fill;
+    r.w = e + 3 < n ? __ldcs(row + e + 3) : fill;
+    return r;
+}
+
+// Guided logit in fp32: subtract, fused multiply-add, divide (three correctly rounded steps).
+__device__ __forceinline__ float guided(float c, float u, float s, float T, int &flags)
+{
+    const bool bad_c = (c != c) || c == CUDART_INF_F, bad_u = (u != u) || u == CUDART_INF_F;
+    if (bad_c || bad_u) flags |= HAWK_DEV_NONFINITE;
+    if (bad_c || bad_u || c == -CUDART_INF_F || u == -CUDART_INF_F) return -CUDART_INF_F;
+    float r = __fdiv_rn(__fmaf_rn(s, __fsub_rn(c, u), u), T);
+    if ((r != r) || r == CUDART_INF_F) {
+        flags |= HAWK_DEV_NONFINITE;
+        r = -CUDART_INF_F;
+    }
+    return r;
+}
+
+template <int NT>
+struct Scratch {
+    float f[3][32];
+    int i[32];
+    float scan[33];
+};
+
+template <int NT>
+__device__ __forceinline__ void block_minmaxcount(float &mx, float &mn, int &cnt, Scratch<NT> &s)
+{
+    constexpr int NW = NT / 32;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+        mn = fminf(mn, __shfl_xor_sync(0xffffffffu, mn, o));
+        cnt += __shfl_xor_sync(0xffffffffu, cnt, o);
+    }
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    __syncthreads();
+    if (lane == 0) {
+        s.f[0][warp] = mx;
+        s.f[1][warp] = mn;
+        s.i[warp] = cnt;
+    }
+    __syncthreads();
+    mx = lane < NW ? s.f[0][lane] : -CUDART_INF_F;
+    mn = lane < NW ? s.f[1][lane] : CUDART_INF_F;
+    cnt = lane < NW ? s.i[lane] : 0;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+        mn = fminf(mn, __shfl_xor_sync(0xffffffffu, mn, o));
+        cnt += __shfl_xor_sync(0xffffffffu, cnt, o);
+    }
+}
+
+template <int NT>
+__device__ __forceinline__ float block_sum(float v, Scratch<NT> &s)
+{
+    constexpr int NW = NT / 32;
+    v = hawk::warp_sum(v);
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    __syncthreads();
+    if (lane == 0) s.f[0][warp] = v;
+    __syncthreads();
+    v = lane < NW ? s.f[0][lane] : 0.f;
+    return hawk::warp_sum(v);
+}
+
+// Exclusive prefix sum over the block in thread order; *total receives the block sum.
+template <int NT, class T>
+__device__ __forceinline__ T block_exclusive_scan(T v, T *scratch33, T *total)
+{
+    constexpr int NW = NT / 32;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    T incl = v;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        T up = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += up;
+    }
+    __syncthreads();
+    if (lane == 31) scratch33[warp] = incl;
+    __syncthreads();
+    if (warp == 0) {
+        T w = lane < NW ? scratch33[lane] : T(0);
+        T wi = w;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            T up = __shfl_up_sync(0xffffffffu, wi, o);
+            if (lane >= o) wi += up;
+        }
+        scratch33[lane] = wi - w;
+        if (lane == 31) scratch33[32] = wi;
+    }
+    __syncthreads();
+    *total = scratch33[32];
+    return scratch33[warp] + (incl - v);
+}
+
+template <int NT, int VPT>
+__global__ void __launch_bounds__(NT) accept_rows_kernel(const AcceptParams P)
+{
+    constexpr int NW = NT / 32;
+    constexpr int BPT = kBins / NT;  // histogram bins per thread
+    static_assert(kBins % NT == 0 && BPT >= 1, "bins must split evenly over the block");
+    static_assert(VPT * NW <= NT, "warp totals of the scan must fit one block-wide scan");
+
+    __shared__ int s_hist[kBins];
+    __shared__ float s_cand[kCandMax];
+    __shared__ Scratch<NT> s_red;
+    __shared__ int s_iscan[33];
+    __shared__ float s_wt[VPT * NW];
+    __shared__ float s_wbase[VPT * NW];
+    __shared__ int s_ncand, s_bin, s_above, s_tok;
+    __shared__ float s_tau, s_px;
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int row = blockIdx.x;  // position-major: all rows of position 0 first
+    const int i = row / P.B, b = row - i * P.B;
+    const bool bonus = (i == P.K);
+    const int n = P.n;
+    const bool vec_ok = P.vec_ok != 0;
+    const float *lc = P.logits + (static_cast<size_t>(b) * P.rows + i) * P.V + P.v_begin;
+    const float *lu = P.logits + (static_cast<size_t>(P.B + b) * P.rows + i) * P.V + P.v_begin;
+    const float *qrow = bonus ? nullptr : P.q + (static_cast<size_t>(b) * P.K + i) * P.V + P.v_begin;
+    int flags = 0;
+
+    // draft id, its q and the uniforms: issued early so the latency hides behind the row load
+    int xd = 0;
+    float qx = 0.f, u_acc = 0.f;
+    if (!bonus) {
+        xd = P.draft[b * P.K + i];
+        if (xd < P.v_begin || xd >= P.v_begin + n) {
+            flags |= HAWK_DEV_BAD_DRAFT;
+            xd = xd < P.v_begin ? P.v_begin : P.v_begin + n - 1;
+        }
+        xd -= P.v_begin;
+        qx = qrow[xd];
+        u_acc = P.u_acc[b * P.K + i];
+    }
+    const float u_res = P.u_res[b * (P.K + 1) + i];
+
+    // ---- read both logit rows once, combine into registers
+    float x[VPT][4];
+    float mx = -CUDART_INF_F, mn = CUDART_INF_F;
+    int cnt = 0;
+#pragma unroll
+    for (int j = 0; j < VPT; ++j) {
+        const int e0 = 4 * (j * NT + tid);
+        if (e0 < n) {
+            const float4 c4 = load4(lc, e0, n, vec_ok, -CUDART_INF_F);
+            const float4 u4 = load4(lu, e0, n, vec_ok, -CUDART_INF_F);
+            int fl = 0;
+            x[j][0] = guided(c4.x, u4.x, P.cfg_scale, P.temperature, fl);
+            x[j][1] = e0 + 1 < n ? guided(c4.y, u4.y, P.cfg_scale, P.temperature, fl) : -CUDART_INF_F;
+            x[j][2] = e0 + 2 < n ? guided(c4.z, u4.z, P.cfg_scale, P.temperature, fl) : -CUDART_INF_F;
+            x[j][3] = e0 + 3 < n ? guided(c4.w, u4.w, P.cfg_scale, P.temperature, fl) : -CUDART_INF_F;
+            flags |= fl;
+        } else {
+            x[j][0] = x[j][1] = x[j][2] = x[j][3] = -CUDART_INF_F;
+        }
+#pragma unroll
+        for (int c = 0; c < 4; ++c)
+            if (x[j][c] > -CUDART_INF_F) {
+                mx = fmaxf(mx, x[j][c]);
+                mn = fminf(mn, x[j][c]);
+                ++cnt;
+            }
+    }
+    block_minmaxcount<NT>(mx, mn, cnt, s_red);
+
+    if (flags && P.dev_status) atomicOr(P.dev_status, flags);
+
+    if (cnt == 0) {  // nothing has mass: p == 0 everywhere, the draft is rejected, no token exists
+        if (P.p_debug) {
+            float *pd = P.p_debug + (static_cast<size_t>(b) * P.rows + i) * P.V + P.v_begin;
+            for (int e = tid; e < n; e += NT) pd[e] = 0.f;
+        }
+        if (tid == 0) P.row_out[b * P.rows + i] = ROW_REJECTED_NO_TOKEN;
+        return;
+    }
+
+    // ---- top-k threshold: the top_k-th largest finite value (exact; ties at it are all kept)
+    float tau = -CUDART_INF_F;
+    if (P.top_k > 0 && P.top_k < cnt) {
+        float lo = mn, hi = mx;
+        int k = P.top_k;
+        for (int round = 0; round < kMaxRounds; ++round) {
+            if (!(hi > lo)) {
+                tau = hi;
+                break;
+            }
+            const float scale = static_cast<float>(kBins) / (hi - lo);
+            for (int t = tid; t < kBins; t += NT) s_hist[t] = 0;
+            if (tid == 0) s_ncand = 0;
+            __syncthreads();
+#pragma unroll
+            for (int j = 0; j < VPT; ++j)
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    const float v = x[j][c];
+                    if (v >= lo && v <= hi) {
+                        const int bin = min(kBins - 1, static_cast<int>((hi - v) * scale));
+                        atomicAdd(&s_hist[bin], 1);
+                    }
+                }
+            __syncthreads();
+            int local = 0;
+#pragma unroll
+            for (int t = 0; t < BPT; ++t) local += s_hist[tid * BPT + t];
+            int total;
+            const int excl = block_exclusive_scan<NT, int>(local, s_iscan, &total);
+            if (excl < k && k <= excl + local) {
+                int run = excl;
+#pragma unroll
+                for (int t = 0; t < BPT; ++t) {
+                    const int h = s_hist[tid * BPT + t];
+                    if (run < k && k <= run + h) {
+                        s_bin = tid * BPT + t;
+                        s_above = run;
+                    }
+                    run += h;
+                }
+            }
+            __syncthreads();
+            const int bstar = s_bin, kk = k - s_above, C = s_hist[bstar];
+            if (C <= kCandMax) {
+#pragma unroll
+                for (int j = 0; j < VPT; ++j)
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) {
+                        const float v = x[j][c];
+                        if (v >= lo && v <= hi) {
+                            const int bin = min(kBins - 1, static_cast<int>((hi - v) * scale));
+                            if (bin == bstar) s_cand[atomicAdd(&s_ncand, 1)] = v;
+                        }
+                    }
+                __syncthreads();
+                for (int t = tid; t < C; t += NT) {
+                    const float v = s_cand[t];
+                    int gt = 0, ge = 0;
+                    for (int m = 0; m < C; ++m) {
+                        const float w = s_cand[m];
+                        gt += w > v;
+                        ge += w >= v;
+                    }
+                    if (gt < kk && kk <= ge) s_tau = v;
+                }
+                __syncthreads();
+                tau = s_tau;
+                break;
+            }
+            // too many candidates share the bin: narrow the range to that bin's values and repeat
+            float nmx = -CUDART_INF_F, nmn = CUDART_INF_F;
+            int dummy = 0;
+#pragma unroll
+            for (int j = 0; j < VPT; ++j)
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    const float v = x[j][c];
+                    if (v >= lo && v <= hi) {
+                        const int bin = min(kBins - 1, static_cast<int>((hi - v) * scale));
+                        if (bin == bstar) {
+                            nmx = fmaxf(nmx, v);
+                            nmn = fminf(nmn, v);
+                        }
+                    }
+                }
+            block_minmaxcount<NT>(nmx, nmn, dummy, s_red);
+            lo = nmn;
+            hi = nmx;
+            k = kk;
+            if (round == kMaxRounds - 1) tau = hi;  // unreachable for fp32 ranges; keeps tau defined
+        }
+    }
+
+    // ---- softmax over what is kept: x becomes exp(l - max), unnormalised
+    constexpr float kLog2e = 1.4426950408889634f;
+    float zsum = 0.f;
+#pragma unroll
+    for (int j = 0; j < VPT; ++j)
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+            const float v = x[j][c];
+            const float e = (v >= tau && v > -CUDART_INF_F) ? hawk::fast_exp2((v - mx) * kLog2e) : 0.f;
+            x[j][c] = e;
+            zsum += e;
+        }
+    const float Z = block_sum<NT>(zsum, s_red);
+    const float invZ = 1.0f / Z;
+
+    if (P.p_debug) {
+        float *pd = P.p_debug + (static_cast<size_t>(b) * P.rows + i) * P.V + P.v_begin;
+#pragma unroll
+        for (int j = 0; j < VPT; ++j)
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                const int e = 4 * (j * NT + tid) + c;
+                if (e < n) pd[e] = x[j][c] * invZ;
+            }
+    }
+
+    // ---- acceptance test on the draft token
+    if (!bonus) {
+#pragma unroll
+        for (int j = 0; j < VPT; ++j)
+#pragma unroll
+            for (int c = 0; c < 4; ++c)
+                if (4 * (j * NT + tid) + c == xd) s_px = x[j][c] * invZ;
+        __syncthreads();
+        const float px = s_px;
+        const bool accepted = static_cast<double>(u_acc) * static_cast<double>(qx) < static_cast<double>(px);
+        if (accepted) {
+            if (tid == 0) P.row_out[b * P.rows + i] = ROW_ACCEPTED;
+            return;
+        }
+    }
+
+    // ---- rejected (or bonus row): inverse-CDF draw from max(0, p - q), or from p itself
+    bool use_q = !bonus;
+    for (int attempt = 0; attempt < 2; ++attempt) {
+        float sj[VPT];
+#pragma unroll
+        for (int j = 0; j < VPT; ++j) {
+            const int e0 = 4 * (j * NT + tid);
+            float4 q4 = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (use_q && e0 < n) q4 = load4(qrow, e0, n, vec_ok, 0.f);
+            const float r0 = fmaxf(0.f, x[j][0] * invZ - q4.x), r1 = fmaxf(0.f, x[j][1] * invZ - q4.y);
+            const float r2 = fmaxf(0.f, x[j][2] * invZ - q4.z), r3 = fmaxf(0.f, x[j][3] * invZ - q4.w);
+            sj[j] = ((r0 + r1) + r2) + r3;
+        }
+        float incl[VPT];
+#pragma unroll
+        for (int j = 0; j < VPT; ++j) {
+            float v = sj[j];
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const float up = __shfl_up_sync(0xffffffffu, v, o);
+                if (lane >= o) v += up;
+            }
+            incl[j] = v;
+            if (lane == 31) s_wt[j * NW + warp] = v;
+        }
+        __syncthreads();
+        float total;
+        {
+            const float v = tid < VPT * NW ? s_wt[tid] : 0.f;
+            const float ex = block_exclusive_scan<NT, float>(v, s_red.scan, &total);
+            if (tid < VPT * NW) s_wbase[tid] = ex;
+            if (tid == 0) s_tok = 0x7fffffff;
+        }
+        __syncthreads();
+        if (use_q && !(total > 0.f)) {  // p <= q everywhere: draw from p with the same uniform
+            use_q = false;
+            continue;
+        }
+        const float t = u_res * total;
+        // pass 0: elements where the running sum crosses t; pass 1 (only if the block-wide sums
+        // disagree at a thread boundary): the first element whose running sum exceeds t
+        for (int pass = 0; pass < 2; ++pass) {
+#pragma unroll
+            for (int j = 0; j < VPT; ++j) {
+                const float excl = s_wbase[j * NW + warp] + (incl[j] - sj[j]);
+                const bool look = pass == 0 ? (excl <= t && excl + sj[j] > t) : (excl + sj[j] > t);
+                if (look) {
+                    const int e0 = 4 * (j * NT + tid);
+                    float4 q4 = make_float4(0.f, 0.f, 0.f, 0.f);
+                    if (use_q && e0 < n) q4 = load4(qrow, e0, n, vec_ok, 0.f);
+                    const float r0 = fmaxf(0.f, x[j][0] * invZ - q4.x), r1 = fmaxf(0.f, x[j][1] * invZ - q4.y);
+                    const float r2 = fmaxf(0.f, x[j][2] * invZ - q4.z), r3 = fmaxf(0.f, x[j][3] * invZ - q4.w);
+                    const float c0 = excl + r0, c1 = excl + (r0 + r1), c2 = excl + ((r0 + r1) + r2);
+                    const float c3 = excl + (((r0 + r1) + r2) + r3);
+                    int hit = -1;  // an id without mass is never drawn
+                    if (r0 > 0.f && c0 > t) hit = 0;
+                    else if (r1 > 0.f && c1 > t) hit = 1;
+                    else if (r2 > 0.f && c2 > t) hit = 2;
+                    else if (r3 > 0.f && c3 > t) hit = 3;
+                    if (hit >= 0) atomicMin(&s_tok, e0 + hit);
+                }
+            }
+            __syncthreads();
+            if (s_tok != 0x7fffffff) break;
+            __syncthreads();
+        }
+        int tok = s_tok;
+        if (tok == 0x7fffffff) {  // rounding left no running sum above t: the last id with mass
+            __syncthreads();
+            if (tid == 0) s_tok = -1;
+            __syncthreads();
+#pragma unroll
+            for (int j = 0; j < VPT; ++j) {
+                const int e0 = 4 * (j * NT + tid);
+                if (sj[j] > 0.f) {
+                    float4 q4 = make_float4(0.f, 0.f, 0.f, 0.f);
+                    if (use_q && e0 < n) q4 = load4(qrow, e0, n, vec_ok, 0.f);
+                    const float r[4] = {x[j][0] * invZ - q4.x, x[j][1] * invZ - q4.y, x[j][2] * invZ - q4.z,
+                                        x[j][3] * invZ - q4.w};
+                    int last = -1;
+#pragma unroll
+                    for (int c = 0; c < 4; ++c)
+                        if (r[c] > 0.f) last = e0 + c;
+                    if (last >= 0) atomicMax(&s_tok, last);
+                }
+            }
+            __syncthreads();
+            tok = s_tok;
+        }
+        if (tid == 0) P.row_out[b * P.rows + i] = tok >= 0 ? P.v_begin + tok : ROW_REJECTED_NO_TOKEN;
+        return;
+    }
+}
+
+// One thread per sequence: the first rejected row decides accept_len and the correction token.
+__global__ void accept_finalize_kernel(const int32_t *row_out, int B, int K, int rows, int32_t *accept_len,
+                                       int32_t *out_token)
+{
+    const int b = blockIdx.x * blockDim.x + threadIdx.x;
+    if (b >= B) return;
+    int len = K, tok = -1;
+    for (int i = 0; i < K; ++i) {
+        const int r = row_out[b * rows + i];
+        if (r != ROW_ACCEPTED) {
+            len = i;
+            tok = r >= 0 ? r : -1;
+            break;
+        }
+    }
+    if (len == K && rows > K) {
+        const int r = row_out[b * rows + K];
+        tok = r >= 0 ? r : -1;
+    }
+    accept_len[b] = len;
+    out_token[b] = tok;
+}
+
+template <int NT, int VPT>
+cudaError_t launch_rows(const AcceptParams &P, int grid, cudaStream_t stream)
+{
+    accept_rows_kernel<NT, VPT><<<grid, NT, 0, stream>>>(P);
+    return cudaGetLastError();
+}
+
+}  // namespace
+
+extern "C" size_t hawk_cfg_accept_workspace_bytes(int B, int K, int V)
+{
+    (void)V;
+    if (B <= 0 || K <= 0) return 0;
+    return static_cast<size_t>(B) * static_cast<size_t>(K + 1) * sizeof(int32_t);
+}
+
+extern "C" hawk_status hawk_cfg_accept(const float *logits, const float *q_probs, const int32_t *draft,
+                                       const float *u_accept, const float *u_resample, int B, int K, int V,
+                                       int v_begin, int v_end, float cfg_scale, float temperature, int top_k,
+                                       int has_bonus_row, int32_t *accept_len, int32_t *out_token, float *p_debug,
+                                       void *workspace, size_t workspace_bytes, int32_t *dev_status,
+                                       hawk_stream_t stream)
+{
+    if (B < 0 || K < 0 || V < 0) return HAWK_ERR_SHAPE;
+    if (B == 0) return HAWK_OK;
+    if (!logits || !q_probs || !draft || !u_accept || !u_resample || !accept_len || !out_token) return HAWK_ERR_NULL;
+    if (v_begin < 0 || v_end > V || v_begin >= v_end) return HAWK_ERR_SHAPE;
+    if (K < 1 || K > 16) return HAWK_ERR_UNSUPPORTED;
+    const int n = v_end - v_begin;
+    if (n > 32768) return HAWK_ERR_UNSUPPORTED;  // one row must fit one block's registers
+    if (!(temperature == temperature) || !(cfg_scale == cfg_scale) || isinf(temperature) || isinf(cfg_scale))
+        return HAWK_ERR_PARAM;
+    if (!(temperature > 0.f)) return HAWK_ERR_PARAM;
+    if (!hawk_host::aligned16(logits) || !hawk_host::aligned16(q_probs) || (p_debug && !hawk_host::aligned16(p_debug)))
+        return HAWK_ERR_ALIGN;
+    const size_t need = hawk_cfg_accept_workspace_bytes(B, K, V);
+    if (!workspace || workspace_bytes < need) return HAWK_ERR_WORKSPACE;
+    if (!hawk_host::aligned16(workspace)) return HAWK_ERR_ALIGN;
+    if (!hawk_host::is_sm100(nullptr)) return HAWK_ERR_UNSUPPORTED;
+
+    AcceptParams P;
+    P.logits = logits;
+    P.q = q_probs;
+    P.draft = draft;
+    P.u_acc = u_accept;
+    P.u_res = u_resample;
+    P.B = B;
+    P.K = K;
+    P.rows = K + (has_bonus_row ? 1 : 0);
+    P.V = V;
+    P.v_begin = v_begin;
+    P.n = n;
+    P.cfg_scale = cfg_scale;
+    P.temperature = temperature;
+    P.top_k = top_k;
+    P.vec_ok = (V % 4 == 0 && v_begin % 4 == 0) ? 1 : 0;
+    P.row_out = static_cast<int32_t *>(workspace);
+    P.p_debug = p_debug;
+    P.dev_status = dev_status;
+
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    const int grid = B * P.rows;
+    cudaError_t err;
+    if (n <= 1024) err = launch_rows<128, 2>(P, grid, st);
+    else if (n <= 4096) err = launch_rows<256, 4>(P, grid, st);
+    else if (n <= 8192) err = launch_rows<512, 4>(P, grid, st);
+    else if (n <= 16384) err = launch_rows<512, 8>(P, grid, st);
+    else err = launch_rows<1024, 8>(P, grid, st);
+    if (err != cudaSuccess) return HAWK_ERR_CUDA;
+    accept_finalize_kernel<<<(B + 127) / 128, 128, 0, st>>>(P.row_out, B, K, P.rows, accept_len, out_token);
+    return cudaGetLastError() == cudaSuccess ? HAWK_OK : HAWK_ERR_CUDA;
+}

@@ -1,0 +1,250 @@
+// hawk_head_proj: logits[m][v] = sum_c x[m][c] * w[v][c] on the 5th-generation tensor cores.
+//
+// The token codebook sits on the MMA's M dimension (128 weight rows per tile) and the token rows on
+// N (16..256), so a handful of draft positions wastes nothing: the instruction's N simply shrinks.
+// Both operands are K-major exactly as stored, so TMA drops [rows][64 columns] boxes with the
+// 128-byte swizzle into shared memory and tcgen05.mma reads them through matrix descriptors.
+//
+// One persistent block per SM, warp-specialised:
+//   warp 0      TMA producer: W box (128 x 64) + X box (BN x 64) per stage, full/empty mbarriers
+//   warp 1      allocates TMEM, issues tcgen05.mma (one lane), commits stages and accumulators
+//   warps 2..5  epilogue: tcgen05.ld of the fp32 accumulator (lane = token id, column = token row),
+//               coalesced 128-byte stores into logits[token][vocab]
+// The accumulator is double-buffered in TMEM so the epilogue of one tile overlaps the MMAs of the next.
+#include "hawk_common.cuh"
+
+namespace {
+
+using namespace hawk;
+
+constexpr int kBM = 128;  // weight rows (token ids) per tile = MMA M
+constexpr int kBK = 64;   // bf16 columns per stage = 128 bytes = one swizzle span
+constexpr int kHeadThreads = 192;
+constexpr int kATileBytes = kBM * kBK * 2;  // 16 KB
+constexpr int kMaxStages = 12;
+constexpr uint32_t kTmemCols = 512;
+
+struct HeadParams {
+    float *logits;
+    int M, hidden, V, v_begin, v_end;
+    int BN;        // token rows per tile (multiple of 16, <= 256)
+    int tiles_m;   // vocab tiles
+    int tiles_n;   // token tiles
+    int stages;
+    int stage_bytes;
+    int32_t *dev_status;
+};
+
+__global__ void __launch_bounds__(kHeadThreads, 1) head_proj_kernel(const __grid_constant__ CUtensorMap map_w,
+                                                                    const __grid_constant__ CUtensorMap map_x,
+                                                                    const HeadParams P)
+{
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    uint64_t *full_bar = reinterpret_cast<uint64_t *>(smem + static_cast<size_t>(P.stages) * P.stage_bytes);
+    uint64_t *empty_bar = full_bar + kMaxStages;
+    uint64_t *acc_full = empty_bar + kMaxStages;  // [2]
+    uint64_t *acc_empty = acc_full + 2;           // [2]
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(acc_empty + 2);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int kblocks = P.hidden / kBK;
+    const int total_tiles = P.tiles_m * P.tiles_n;
+
+    if (tid == 0) {
+        for (int i = 0; i < P.stages; ++i) {
+            mbar_init(&full_bar[i], 1);
+            mbar_init(&empty_bar[i], 1);
+        }
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(&acc_full[i], 1);
+            mbar_init(&acc_empty[i], 4);  // one arrival per epilogue warp
+        }
+        *abort_flag = 0;
+        fence_mbar_init();
+    }
+    if (warp == 1) {
+        tmem_alloc(tmem_slot, kTmemCols);
+        tmem_relinquish();
+    }
+    tcgen05_fence_before();
+    __syncthreads();
+    tcgen05_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp == 0) {
+        // =========================== TMA producer
+        if (lane == 0) {
+            prefetch_tensormap(&map_w);
+            prefetch_tensormap(&map_x);
+            const uint32_t tx_bytes = static_cast<uint32_t>(P.stage_bytes);
+            int st = 0;
+            uint32_t ph = 0;
+            bool ok = true;
+            long long issued = 0;
+            for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+                const int tn = tile % P.tiles_n, tm = tile / P.tiles_n;
+                const int row_w = P.v_begin + tm * kBM, row_x = tn * P.BN;
+                for (int kb = 0; kb < kblocks; ++kb) {
+                    ok = mbar_wait(&empty_bar[st], ph ^ 1u, abort_flag);
+                    if (!ok) break;
+                    uint8_t *a = smem + static_cast<size_t>(st) * P.stage_bytes;
+                    mbar_arrive_expect_tx(&full_bar[st], tx_bytes);
+                    tma_load_2d(a, &map_w, kb * kBK, row_w, &full_bar[st]);
+                    tma_load_2d(a + kATileBytes, &map_x, kb * kBK, row_x, &full_bar[st]);
+                    ++issued;
+                    if (++st == P.stages) {
+                        st = 0;
+                        ph ^= 1u;
+                    }
+                }
+            }
+            if (!ok) {
+                *abort_flag = 1;
+                if (P.dev_status) atomicOr(P.dev_status, HAWK_DEV_TIMEOUT);
+            }
+        }
+    } else if (warp == 1) {
+        // =========================== MMA issuer
+        if (lane == 0) {
+            const uint32_t idesc = umma_idesc_bf16_f32(kBM, P.BN);
+            int st = 0;
+            uint32_t ph = 0;
+            bool ok = true;
+            int it = 0;
+            for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++it) {
+                const int ab = it & 1;
+                const uint32_t acc_ph = (it >> 1) & 1;
+                ok = mbar_wait(&acc_empty[ab], acc_ph ^ 1u, abort_flag);  // epilogue drained this buffer
+                if (!ok) break;
+                tcgen05_fence_after();
+                const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(ab * P.BN);
+                for (int kb = 0; kb < kblocks; ++kb) {
+                    ok = mbar_wait(&full_bar[st], ph, abort_flag);
+                    if (!ok) break;
+                    tcgen05_fence_after();
+                    const uint32_t a_addr = smem_u32(smem + static_cast<size_t>(st) * P.stage_bytes);
+                    const uint64_t da = umma_desc_k_major_sw128(a_addr);
+                    const uint64_t db = umma_desc_k_major_sw128(a_addr + kATileBytes);
+#pragma unroll
+                    for (int k = 0; k < kBK / 16; ++k) {
+                        // 16 bf16 along K = 32 bytes = 2 units of the descriptor's 16-byte address field
+                        umma_bf16(d_tmem, da + static_cast<uint64_t>(2 * k), db + static_cast<uint64_t>(2 * k), idesc,
+                                  (kb | k) != 0 ? 1u : 0u);
+                    }
+                    umma_commit(&empty_bar[st]);  // stage reusable once these MMAs have read it
+                    if (++st == P.stages) {
+                        st = 0;
+                        ph ^= 1u;
+                    }
+                }
+                if (!ok) break;
+                umma_commit(&acc_full[ab]);  // accumulator complete
+            }
+            if (!ok) {
+                *abort_flag = 1;
+                if (P.dev_status) atomicOr(P.dev_status, HAWK_DEV_TIMEOUT);
+            }
+        }
+    } else {
+        // =========================== epilogue warps: TMEM lanes 32*(warp%4) .. +31
+        const int lane_base = (warp & 3) * 32;
+        bool ok = true;
+        int it = 0;
+        for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++it) {
+            const int tn = tile % P.tiles_n, tm = tile / P.tiles_n;
+            const int ab = it & 1;
+            const uint32_t acc_ph = (it >> 1) & 1;
+            ok = mbar_wait(&acc_full[ab], acc_ph, abort_flag);
+            if (!ok) break;
+            tcgen05_fence_after();
+            const int v = P.v_begin + tm * kBM + lane_base + lane;  // this thread's token id
+            const bool v_ok = v < P.v_end;
+            const int n0 = tn * P.BN;
+            const uint32_t taddr = tmem_base + (static_cast<uint32_t>(lane_base) << 16) + static_cast<uint32_t>(ab * P.BN);
+            for (int c = 0; c < P.BN; c += 16) {
+                uint32_t r[16];
+                tmem_ld_32x16(taddr + c, r);
+                tmem_ld_wait();
+                if (v_ok) {
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) {
+                        const int n = n0 + c + j;
+                        if (n < P.M) P.logits[static_cast<size_t>(n) * P.V + v] = __uint_as_float(r[j]);
+                    }
+                }
+            }
+            tcgen05_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&acc_empty[ab]);
+        }
+        if (!ok && lane == 0) {
+            *abort_flag = 1;
+            if (P.dev_status) atomicOr(P.dev_status, HAWK_DEV_TIMEOUT);
+        }
+    }
+
+    tcgen05_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tcgen05_fence_after();
+        tmem_dealloc(tmem_base, kTmemCols);
+    }
+}
+
+}  // namespace
+
+extern "C" hawk_status hawk_head_proj(const void *x, const void *w, float *logits, int M, int hidden, int V,
+                                      int v_begin, int v_end, int32_t *dev_status, hawk_stream_t stream)
+{
+    if (M < 0 || hidden < 0 || V < 0) return HAWK_ERR_SHAPE;
+    if (v_begin < 0 || v_end > V || v_begin > v_end) return HAWK_ERR_SHAPE;
+    if (M == 0 || v_begin == v_end) return HAWK_OK;
+    if (!x || !w || !logits) return HAWK_ERR_NULL;
+    if (hidden < 64 || hidden % 64 != 0) return HAWK_ERR_UNSUPPORTED;
+    if (!hawk_host::aligned16(x) || !hawk_host::aligned16(w) || !hawk_host::aligned16(logits)) return HAWK_ERR_ALIGN;
+    int sm_count = 0;
+    if (!hawk_host::is_sm100(&sm_count)) return HAWK_ERR_UNSUPPORTED;
+
+    HeadParams P;
+    P.logits = logits;
+    P.M = M;
+    P.hidden = hidden;
+    P.V = V;
+    P.v_begin = v_begin;
+    P.v_end = v_end;
+    P.tiles_n = (M + 255) / 256;
+    const int per_tile = (M + P.tiles_n - 1) / P.tiles_n;
+    P.BN = (per_tile + 15) / 16 * 16;
+    P.tiles_m = (v_end - v_begin + kBM - 1) / kBM;
+    P.stage_bytes = kATileBytes + P.BN * kBK * 2;
+    const int smem_budget = 200 * 1024;
+    int stages = smem_budget / P.stage_bytes;
+    if (stages > kMaxStages) stages = kMaxStages;
+    if (stages < 2) return HAWK_ERR_UNSUPPORTED;
+    P.stages = stages;
+    P.dev_status = dev_status;
+
+    CUtensorMap map_w, map_x;
+    if (!hawk_host::encode_bf16_rows_sw128(&map_w, w, static_cast<uint64_t>(V), static_cast<uint64_t>(hidden), kBM,
+                                           true) ||
+        !hawk_host::encode_bf16_rows_sw128(&map_x, x, static_cast<uint64_t>(M), static_cast<uint64_t>(hidden),
+                                           static_cast<uint32_t>(P.BN), true))
+        return HAWK_ERR_CUDA;
+
+    // always ask for enough shared memory that a second block cannot share the SM: each block owns all of TMEM
+    const size_t smem_bytes = 1024 + static_cast<size_t>(stages) * P.stage_bytes + (2 * kMaxStages + 4) * 8 + 64;
+    const size_t smem_req = smem_bytes < 120 * 1024 ? 120 * 1024 : smem_bytes;
+    static bool attr_done = false;
+    if (!attr_done) {
+        if (cudaFuncSetAttribute(head_proj_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) !=
+            cudaSuccess)
+            return HAWK_ERR_CUDA;
+        attr_done = true;
+    }
+    const int total_tiles = P.tiles_m * P.tiles_n;
+    const int grid = total_tiles < sm_count ? total_tiles : sm_count;
+    head_proj_kernel<<<grid, kHeadThreads, smem_req, reinterpret_cast<cudaStream_t>(stream)>>>(map_w, map_x, P);
+    return cudaGetLastError() == cudaSuccess ? HAWK_OK : HAWK_ERR_CUDA;
+}

@@ -1,0 +1,147 @@
+"""GPU parity of hawk_cfg_accept against the oracle (through the C ABI)."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2510_25739_b200 import workloads as wl
+from tests._util import compare_accept, to_dev
+
+pytestmark = pytest.mark.gpu
+
+
+def _run_case(cfg, seed, logits=None, q=None, has_bonus=False, check_p=True, drafts=None):
+    import paper_2510_25739_b200 as hawk
+    if logits is None:
+        logits = wl.make_logits(cfg, seed, has_bonus_row=has_bonus)
+    p, row_flags = oracle.target_probs_rows(logits, cfg.v_begin, cfg.v_end, cfg.cfg_scale, cfg.temperature,
+                                            cfg.top_k)
+    if q is None:
+        q = wl.make_q(cfg, seed, np.nan_to_num(p[:, :cfg.K]))
+    if drafts is None:
+        drafts = wl.draw_drafts(q, seed)
+    u = wl.draw_uniforms(cfg, seed)
+    ora = oracle.cfg_accept(logits, q, drafts, u["u_accept"], u["u_resample"], cfg.v_begin, cfg.v_end,
+                            cfg.cfg_scale, cfg.temperature, cfg.top_k, has_bonus_row=has_bonus)
+    rows = cfg.K + (1 if has_bonus else 0)
+    p_dbg = torch.full((cfg.B, rows, cfg.V), -1.0, dtype=torch.float32, device="cuda") if check_p else None
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    alen, tok = hawk.cfg_accept(to_dev(logits), to_dev(q), to_dev(drafts), to_dev(u["u_accept"]),
+                                to_dev(u["u_resample"]), cfg.v_begin, cfg.v_end, cfg.cfg_scale, cfg.temperature,
+                                cfg.top_k, has_bonus_row=has_bonus, p_debug=p_dbg, dev_status=status)
+    torch.cuda.synchronize()
+    # the kernel examines every row, the oracle's chain stops at the first rejection: expected
+    # device flags are those of all rows
+    bad_draft = ((drafts < cfg.v_begin) | (drafts >= cfg.v_end)).any()
+    assert int(status.item()) == (row_flags | (oracle.FLAG_BAD_DRAFT if bad_draft else 0))
+    res = compare_accept(alen.cpu().numpy(), tok.cpu().numpy(), ora, cfg.K)
+    assert not res["bad"], res["bad"][:10]
+    if check_p:
+        got = p_dbg.cpu().numpy().astype(np.float64)[:, :, cfg.v_begin:cfg.v_end]
+        want = p[:, :, cfg.v_begin:cfg.v_end]
+        np.testing.assert_allclose(got, want, rtol=1e-5, atol=1e-12)
+        # ids outside the valid range are never written
+        if cfg.v_begin > 0:
+            assert (p_dbg[:, :, :cfg.v_begin] == -1).all()
+        if cfg.v_end < cfg.V:
+            assert (p_dbg[:, :, cfg.v_end:] == -1).all()
+    return res, ora
+
+
+SMALL = [
+    # V, v_begin, v_end, top_k, K, B
+    (64, 0, 64, 0, 1, 3),
+    (64, 0, 64, 10, 4, 5),
+    (1000, 0, 1000, 100, 3, 4),
+    (1000, 3, 999, 1, 2, 4),          # unaligned range, greedy-like top-1
+    (4096, 4, 4000, 2000, 5, 3),
+    (5000, 0, 5000, 4999, 2, 2),      # row length not a multiple of the vector width; k = n - 1
+    (16384, 0, 16384, 2000, 6, 4),
+    (16384, 8, 16000, 16000, 2, 2),   # top_k >= valid ids: no filter
+    (20000, 0, 20000, 50, 2, 2),      # more than 16384 ids
+    (65536, 4, 8196, 2000, 3, 2),
+]
+
+
+@pytest.mark.parametrize("V,vb,ve,top_k,K,B", SMALL)
+@pytest.mark.parametrize("bonus", [False, True])
+def test_small_cases(V, vb, ve, top_k, K, B, bonus):
+    cfg = wl.config(2, B=B, K=K, V=V, v_begin=vb, v_end=ve, top_k=top_k, cfg_scale=3.0, H=4, H_kv=4)
+    res, _ = _run_case(cfg, 77 + V + K, has_bonus=bonus)
+    assert res["exempt_accept"] + res["exempt_resample"] <= B
+
+
+@pytest.mark.parametrize("config_id", [1, 2, 3, 4, 5])
+def test_configs_full_size(config_id):
+    cfg = wl.config(config_id)
+    res, ora = _run_case(cfg, wl.seed_for(config_id))
+    assert res["exempt_accept"] + res["exempt_resample"] <= max(2, cfg.B // 8)
+    print(f"config {config_id}: exempt {res['exempt_accept']}+{res['exempt_resample']}, checked {res['checked']}, "
+          f"mean accept_len {ora['accept_len'].mean():.3f}")
+
+
+@pytest.mark.parametrize("alpha", wl.STRESS_ALPHAS)
+def test_stress_alphas(alpha):
+    cfg = wl.config(5, q_alpha=alpha)
+    res, ora = _run_case(cfg, wl.seed_for(5, int(alpha * 10) + 1), check_p=False)
+    if alpha == 1.0:      # q is p rounded to fp32: everything not within rounding of the threshold passes
+        assert (ora["accept_len"] >= 0).all()
+    assert res["exempt_accept"] + res["exempt_resample"] <= cfg.B // 4 or alpha == 1.0
+
+
+def test_stress_disjoint_support():
+    cfg = wl.config(5, q_recipe="disjoint")
+    logits = wl.mask_odd_ids(wl.make_logits(cfg, 5900), cfg)
+    res, ora = _run_case(cfg, 5900, logits=logits)
+    assert (ora["accept_len"] == 0).all()
+
+
+def test_q_equal_p_accepts_everything():
+    cfg = wl.config(2, B=6, K=5)
+    logits = wl.make_logits(cfg, 31)
+    p, _ = oracle.target_probs_rows(logits, 0, cfg.V, cfg.cfg_scale, 1.0, cfg.top_k)
+    q = p.astype(np.float32)
+    import paper_2510_25739_b200 as hawk
+    drafts = wl.draw_drafts(q, 31)
+    ua = np.full((cfg.B, cfg.K), 0.5, np.float32)
+    ur = np.zeros((cfg.B, cfg.K + 1), np.float32)
+    alen, tok = hawk.cfg_accept(to_dev(logits), to_dev(q), to_dev(drafts), to_dev(ua), to_dev(ur), 0, cfg.V,
+                                cfg.cfg_scale, 1.0, cfg.top_k)
+    assert (alen.cpu().numpy() == cfg.K).all() and (tok.cpu().numpy() == -1).all()
+
+
+def test_ties_duplicates_and_masked_rows():
+    """Heavy ties at the top-k threshold, all-equal rows, fully masked rows, -inf and NaN entries."""
+    cfg = wl.config(2, B=4, K=3, V=4096, v_end=4096, top_k=100, cfg_scale=2.0)
+    rng = np.random.default_rng(5)
+    logits = np.round(rng.standard_normal((2 * cfg.B, cfg.K, cfg.V)) * 2).astype(np.float32)  # many exact ties
+    logits[0, 0, :] = 1.0; logits[cfg.B, 0, :] = 1.0            # all equal
+    logits[1, 1, :] = -np.inf                                   # conditional stream fully masked
+    logits[2, 2, 7] = np.nan                                    # flagged, treated as -inf
+    logits[3, 0, 100:4000] = -np.inf
+    q = wl.random_probs(cfg, 5).astype(np.float32)
+    res, ora = _run_case(cfg, 5, logits=logits, q=q)
+    _, flags = oracle.target_probs_rows(logits, 0, cfg.V, 2.0, 1.0, 100)
+    assert flags == oracle.FLAG_NONFINITE
+
+
+def test_out_of_range_draft_is_clamped_and_flagged():
+    cfg = wl.config(2, B=2, K=2, V=1024, v_begin=8, v_end=1000, top_k=0)
+    logits = wl.make_logits(cfg, 9)
+    q = wl.random_probs(cfg, 9).astype(np.float32)
+    drafts = np.array([[2, 500], [1023, 20]], np.int32)
+    res, ora = _run_case(cfg, 9, logits=logits, q=q, drafts=drafts)
+
+
+def test_deterministic_across_runs():
+    import paper_2510_25739_b200 as hawk
+    cfg = wl.config(3)
+    logits = to_dev(wl.make_logits(cfg, 3))
+    q = to_dev(wl.random_probs(cfg, 3).astype(np.float32))
+    d = to_dev(wl.draw_drafts(q.cpu().numpy(), 3)); u = wl.draw_uniforms(cfg, 3)
+    outs = []
+    for _ in range(2):
+        a, t = hawk.cfg_accept(logits, q, d, to_dev(u["u_accept"]), to_dev(u["u_resample"]), 0, cfg.V,
+                               cfg.cfg_scale, 1.0, cfg.top_k)
+        outs.append((a.cpu().numpy().copy(), t.cpu().numpy().copy()))
+    assert (outs[0][0] == outs[1][0]).all() and (outs[0][1] == outs[1][1]).all()
