@@ -1,0 +1,527 @@
+#!/usr/bin/env python
+"""Benchmark of the verify step (attention -> head projection -> CFG accept) on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config C] [--impl reference]
+
+One "step" is one pass of the whole verify path over one batch of synthetic inputs shaped like
+workload C (default 2: LlamaGen-XL-shaped, KV length 1144).  Rank 0 prints ONE JSON line.
+
+* value            verified draft positions per second, inputs resident in HBM, whole job (all ranks);
+                   each step is a CUDA-graph replay of the three C-ABI calls.
+* e2e              same metric through hawk_verify_step_host: pinned host buffers, host->device
+                   copies of the step's inputs and device->host copy of the results inside the
+                   timed region.
+* roofline         the dominant kernel (attention), timed with CUDA events inside the timed steps.
+* cpu_baseline     the CPU oracle timed on the host cores on a bounded sample (rank 0, N=1 only).
+* --impl reference times that same oracle as the reference arm.
+
+Inputs rotate over enough replicas that consecutive steps never find their data in L2.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import sys
+import threading
+import time
+from dataclasses import replace
+from pathlib import Path
+
+import numpy as np
+
+ROOT = Path(__file__).resolve().parent
+if str(ROOT) not in sys.path:
+    sys.path.insert(0, str(ROOT))
+
+from paper_2510_25739_b200 import workloads as wl  # noqa: E402
+
+METRIC = "verified draft positions/sec per B200 (verify step)"
+UNIT = "positions/s"
+L2_BYTES = 126 * 1024 * 1024
+
+
+def measured_peaks():
+    p = ROOT / "MEASURED_PEAKS.json"
+    if p.exists():
+        d = json.loads(p.read_text())
+        return dict(hbm_gbs=float(d["hbm_gbs"]), bf16_tflops=float(d["bf16_tflops"]),
+                    bf16_tflops_sustained=float(d.get("bf16_tflops_sustained", d["bf16_tflops"])), source="measured")
+    return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, bf16_tflops_sustained=1400.0, source="fallback")
+
+
+# ------------------------------------------------------------------------------------------ bytes / flops
+def attn_bytes(cfg) -> int:
+    """Algorithmic HBM bytes of one attention launch: K and V rows every query can see, plus Q and O."""
+    kv = cfg.S * cfg.H_kv * (cfg.L + cfg.K) * cfg.D * 2 * 2
+    qo = 2 * cfg.S * cfg.K * cfg.H * cfg.D * 2
+    return kv + qo
+
+
+def head_bytes(cfg) -> int:
+    return cfg.V_valid * cfg.hidden * 2 + cfg.M * cfg.hidden * 2 + cfg.M * cfg.V_valid * 4
+
+
+def head_flops(cfg) -> int:
+    return 2 * cfg.M * cfg.hidden * cfg.V_valid
+
+
+def accept_bytes(cfg, q_rows_read: int) -> int:
+    return 2 * cfg.B * cfg.K * cfg.V_valid * 4 + q_rows_read * cfg.V_valid * 4
+
+
+# ------------------------------------------------------------------------------------------ clocks
+class ClockSampler:
+    """Samples SM clock and throttle reasons through NVML while the timed region runs."""
+
+    def __init__(self, index: int, uuid: str = "", period_s: float = 0.05):
+        self.index, self.period = index, period_s
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop = threading.Event()
+        self._thread = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = None
+            if uuid:
+                try:
+                    self.h = pynvml.nvmlDeviceGetHandleByUUID(uuid)
+                except Exception:
+                    self.h = None
+            if self.h is None:
+                self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+        except Exception:
+            self.nv = None
+
+    def _once(self):
+        nv = self.nv
+        self.samples.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+        try:
+            r = nv.nvmlDeviceGetCurrentClocksEventReasons(self.h)
+        except Exception:
+            r = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+        names = {
+            "sw_power_cap": getattr(nv, "nvmlClocksEventReasonSwPowerCap", 0x4),
+            "hw_slowdown": getattr(nv, "nvmlClocksEventReasonHwSlowdown", 0x8),
+            "sw_thermal_slowdown": getattr(nv, "nvmlClocksEventReasonSwThermalSlowdown", 0x20),
+            "hw_thermal_slowdown": getattr(nv, "nvmlClocksEventReasonHwThermalSlowdown", 0x40),
+            "hw_power_brake": getattr(nv, "nvmlClocksEventReasonHwPowerBrakeSlowdown", 0x80),
+        }
+        for k, bit in names.items():
+            if r & bit:
+                self.reasons.add(k)
+
+    def _run(self):
+        while not self._stop.is_set():
+            try:
+                self._once()
+            except Exception:
+                pass
+            self._stop.wait(self.period)
+
+    def start(self):
+        if self.nv is None:
+            return
+        self._thread = threading.Thread(target=self._run, daemon=True)
+        self._thread.start()
+
+    def stop(self):
+        if self._thread:
+            self._stop.set()
+            self._thread.join()
+            self._thread = None
+            self._stop.clear()
+
+    def summary(self):
+        if not self.samples:
+            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": 0}
+        return {"sm_mhz": statistics.median(self.samples), "sm_max_mhz": self.max_mhz,
+                "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+# ------------------------------------------------------------------------------------------ inputs
+def synth_q(cfg, x, w, gen, torch):
+    """Draft probabilities q = a*p + (1-a)*r for the bench (input synthesis with library ops only).
+
+    p is the target distribution of the logits the head will produce for these x and w (matmul, top-k
+    threshold and softmax by torch), r a random dense distribution over the valid ids.
+    """
+    lg = (x.float() @ w[cfg.v_begin:cfg.v_end].float().t()).view(cfg.S, cfg.K, cfg.V_valid)
+    g = torch.addcmul(lg[cfg.B:], lg[:cfg.B] - lg[cfg.B:], torch.tensor(cfg.cfg_scale, device=x.device))
+    g = g / cfg.temperature
+    if 0 < cfg.top_k < cfg.V_valid:
+        tau = torch.topk(g, cfg.top_k, dim=-1).values[..., -1:]
+        g = torch.where(g >= tau, g, torch.full_like(g, float("-inf")))
+    p = torch.softmax(g.double(), dim=-1)
+    r = torch.softmax(torch.randn(p.shape, generator=gen, device=x.device, dtype=torch.float64), dim=-1)
+    if cfg.q_recipe == "own":
+        qv = r
+    elif cfg.q_recipe == "mix_row_uniform":
+        a = 0.3 + 0.65 * torch.rand((cfg.B, cfg.K, 1), generator=gen, device=x.device, dtype=torch.float64)
+        qv = a * p + (1 - a) * r
+    else:
+        qv = cfg.q_alpha * p + (1 - cfg.q_alpha) * r
+    q = torch.zeros((cfg.B, cfg.K, cfg.V), dtype=torch.float32, device=x.device)
+    q[..., cfg.v_begin:cfg.v_end] = qv.float()
+    draft = torch.multinomial(qv.view(-1, cfg.V_valid).float(), 1, generator=gen).view(cfg.B, cfg.K) + cfg.v_begin
+    return q, draft.int()
+
+
+class Replica:
+    """Device-resident inputs, intermediates and outputs of one step."""
+
+    def __init__(self, cfg, seed, torch, hawk):
+        dev = torch.device("cuda")
+        gen = torch.Generator(device=dev)
+        gen.manual_seed(seed)
+        S, K, H, Hkv, D, Lc = cfg.S, cfg.K, cfg.H, cfg.H_kv, cfg.D, cfg.L_cap
+        bf = torch.bfloat16
+        self.q = torch.randn((S, K, H, D), generator=gen, device=dev).to(bf)
+        self.k_cache = torch.randn((S, Hkv, Lc, D), generator=gen, device=dev).to(bf)
+        self.v_cache = torch.randn((S, Hkv, Lc, D), generator=gen, device=dev).to(bf)
+        self.prefix_len = torch.full((S,), cfg.L, dtype=torch.int32, device=dev)
+        self.x = torch.randn((cfg.M, cfg.hidden), generator=gen, device=dev).to(bf)
+        self.w = (0.02 * torch.randn((cfg.V, cfg.hidden), generator=gen, device=dev)).to(bf)
+        self.q_probs, self.draft = synth_q(cfg, self.x, self.w, gen, torch)
+        self.u_accept = torch.rand((cfg.B, K), generator=gen, device=dev)
+        self.u_resample = torch.rand((cfg.B, K + 1), generator=gen, device=dev)
+        self.attn_out = torch.empty((S, K, H * D), dtype=bf, device=dev)
+        self.logits = torch.zeros((cfg.M, cfg.V), dtype=torch.float32, device=dev)
+        self.accept_len = torch.empty(cfg.B, dtype=torch.int32, device=dev)
+        self.out_token = torch.empty(cfg.B, dtype=torch.int32, device=dev)
+        self.status = torch.zeros(1, dtype=torch.int32, device=dev)
+        ws = hawk.verify_attn_workspace_bytes(S, K, H, Hkv, D, cfg.L)
+        self.attn_ws = torch.empty(max(ws, 16), dtype=torch.uint8, device=dev)
+        self.attn_split = ws > 0
+        self.acc_ws = torch.empty(max(hawk.cfg_accept_workspace_bytes(cfg.B, K, cfg.V), 16), dtype=torch.uint8,
+                                  device=dev)
+        self.sm_scale = 1.0 / float(np.sqrt(D))
+
+    def bytes(self) -> int:
+        ts = (self.q, self.k_cache, self.v_cache, self.x, self.w, self.q_probs, self.logits)
+        return sum(t.numel() * t.element_size() for t in ts)
+
+
+def run_attn(cfg, r, hawk):
+    hawk.verify_attn(r.q, r.k_cache, r.v_cache, r.prefix_len, cfg.L, r.sm_scale, out=r.attn_out,
+                     workspace=r.attn_ws, dev_status=r.status)
+
+
+def run_head(cfg, r, hawk):
+    hawk.head_proj(r.x, r.w, cfg.v_begin, cfg.v_end, logits=r.logits, dev_status=r.status)
+
+
+def run_accept(cfg, r, hawk):
+    hawk.cfg_accept(r.logits.view(cfg.S, cfg.K, cfg.V), r.q_probs, r.draft, r.u_accept, r.u_resample, cfg.v_begin,
+                    cfg.v_end, cfg.cfg_scale, cfg.temperature, cfg.top_k, accept_len=r.accept_len,
+                    out_token=r.out_token, workspace=r.acc_ws, dev_status=r.status)
+
+
+def make_event(torch):
+    try:
+        return torch.cuda.Event(enable_timing=True, external=True), True
+    except TypeError:
+        return torch.cuda.Event(enable_timing=True), False
+
+
+# ------------------------------------------------------------------------------------------ CPU oracle leg
+def oracle_sample(cfg, seed, reps):
+    """Times the CPU oracle (as it stands) on `reps` full steps of the workload; returns positions/s."""
+    import oracle
+    a = wl.make_attn_inputs(cfg, seed)
+    h = wl.make_head_inputs(cfg, seed)
+    q = wl.make_q(replace(cfg, q_recipe="own"), seed, None)   # timing only: any dense q will do
+    drafts = wl.draw_drafts(q, seed)
+    u = wl.draw_uniforms(cfg, seed)
+    oracle.build()
+    t0 = time.perf_counter()
+    for _ in range(reps):
+        oracle.verify_attn(a["q"], a["k_cache"], a["v_cache"], a["prefix_len"], a["sm_scale"])
+        lg = oracle.head_proj(h["x"], h["w"], cfg.v_begin, cfg.v_end, fill=0.0)
+        oracle.cfg_accept(lg.reshape(cfg.S, cfg.K, cfg.V), q, drafts, u["u_accept"], u["u_resample"], cfg.v_begin,
+                          cfg.v_end, cfg.cfg_scale, cfg.temperature, cfg.top_k, diagnostics=False)
+    dt = time.perf_counter() - t0
+    return cfg.B * cfg.K * reps / dt, dt, oracle.threads()
+
+
+def workload_name(cfg, cid):
+    return (f"config {cid} ({cfg.name}): B={cfg.B} x2 CFG streams, K={cfg.K}, {cfg.H} heads x {cfg.D}, "
+            f"hidden {cfg.hidden}, KV length {cfg.L}, vocab {cfg.V} ({cfg.V_valid} valid), "
+            f"cfg {cfg.cfg_scale}, top-k {cfg.top_k}, T {cfg.temperature}")
+
+
+def reference_arm(args, cfg, cid):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    _, t1, cores = oracle_sample(cfg, wl.seed_for(cid), 1)          # also warms the build and the page cache
+    steps = max(1, min(args.steps, int(120.0 / max(t1, 1e-3))))      # the whole run ends within minutes
+    total = 0.0
+    for _ in range(steps):
+        _, dt, cores = oracle_sample(cfg, wl.seed_for(cid), 1)
+        total += dt
+    value = cfg.B * cfg.K * steps / total
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": steps,
+        "warmup": 1, "ms_per_step": 1e3 * total / steps, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": workload_name(cfg, cid), "note": "CPU oracle, one full step of the workload per step"},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle",
+                         "sample": f"{steps} full steps of the workload"},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+# ------------------------------------------------------------------------------------------ main arm
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=2000)
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--config", type=int, default=2, help="workload id 1..5 (default 2: LlamaGen-XL-shaped)")
+    ap.add_argument("--impl", default="hawk", choices=["hawk", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    args = ap.parse_args()
+    cid = args.config
+    cfg = wl.config(cid)
+    if args.impl == "reference":
+        reference_arm(args, cfg, cid)
+        return
+
+    import torch
+    import paper_2510_25739_b200 as hawk
+    from paper_2510_25739_b200 import binding
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device; there is no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    hawk.load_library()
+    W = max(args.warmup, 3)
+    K_steps = max(args.steps, 1)
+
+    # ---- replicas: enough bytes that a step never finds its inputs in L2
+    first = Replica(cfg, 1000 * cid + 17 * rank, torch, hawk)
+    n_rep = max(2, -(-3 * L2_BYTES // first.bytes()))
+    n_rep = min(n_rep, 64)
+    reps = [first] + [Replica(cfg, 1000 * cid + 17 * rank + 101 * i, torch, hawk) for i in range(1, n_rep)]
+    stream = torch.cuda.Stream()
+    launches_per_step = (2 if first.attn_split else 1) + 1 + 2
+
+    # ---- one CUDA graph per replica: [ev0] attn [ev1] head accept
+    graphs, evs = [], []
+    external_events = True
+    with torch.cuda.stream(stream):
+        for r in reps:                       # warm the kernels (function attributes are set on first use)
+            run_attn(cfg, r, hawk); run_head(cfg, r, hawk); run_accept(cfg, r, hawk)
+        stream.synchronize()
+        for r in reps:
+            e0, ext0 = make_event(torch)
+            e1, ext1 = make_event(torch)
+            external_events &= ext0 and ext1
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=stream):
+                if external_events:
+                    e0.record()
+                run_attn(cfg, r, hawk)
+                if external_events:
+                    e1.record()
+                run_head(cfg, r, hawk)
+                run_accept(cfg, r, hawk)
+            graphs.append(g)
+            evs.append((e0, e1))
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    try:
+        uuid = "GPU-" + str(torch.cuda.get_device_properties(local_rank).uuid)
+    except Exception:
+        uuid = ""
+    sampler = ClockSampler(local_rank, uuid)
+    start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    attn_ms = []
+    with torch.cuda.stream(stream):
+        for i in range(W):
+            graphs[i % n_rep].replay()
+        barrier()
+        sampler.start()
+        start.record(stream)
+        for i in range(K_steps):
+            graphs[i % n_rep].replay()
+        stop.record(stream)
+        barrier()
+        sampler.stop()
+    elapsed_ms = start.elapsed_time(stop)
+    if dist is not None:
+        t = torch.tensor([elapsed_ms], device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        elapsed_ms = float(t.item())
+    ms_per_step = elapsed_ms / K_steps
+    positions = cfg.B * cfg.K
+    value = positions * world / (ms_per_step * 1e-3)
+    status = int(sum(int(r.status.item()) for r in reps))
+
+    # ---- dominant kernel: attention, from the events recorded inside the timed graphs (last round of
+    # replays), else from a loop of attention-only launches on the same stream
+    timing_mode = "events inside the timed step graphs"
+    if external_events:
+        try:
+            attn_ms = [e0.elapsed_time(e1) for (e0, e1) in evs[: min(n_rep, K_steps)]]
+        except Exception:
+            attn_ms = []
+    if not attn_ms:
+        timing_mode = "attention-only loop (graph event nodes unavailable)"
+        with torch.cuda.stream(stream):
+            a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            n = max(50, min(K_steps, 500))
+            for i in range(5):
+                run_attn(cfg, reps[i % n_rep], hawk)
+            stream.synchronize()
+            a0.record(stream)
+            for i in range(n):
+                run_attn(cfg, reps[i % n_rep], hawk)
+            a1.record(stream)
+            stream.synchronize()
+            attn_ms = [a0.elapsed_time(a1) / n]
+    peaks = measured_peaks()
+    attn_s = statistics.mean(attn_ms) * 1e-3
+    achieved = attn_bytes(cfg) / attn_s / 1e9
+    roofline = {"kernel": "hawk_verify_attn", "bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"],
+                "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"], "peak_source": f"of {peaks['source']}",
+                "traffic": None, "us_per_launch": attn_s * 1e6, "algorithmic_bytes": attn_bytes(cfg),
+                "timing": timing_mode}
+
+    # ---- per-kernel loops (each kernel alone, rotating replicas) for the stage breakdown
+    kernels = {}
+    with torch.cuda.stream(stream):
+        for name, fn in (("attn", run_attn), ("head", run_head), ("accept", run_accept)):
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=stream):
+                for r in reps:
+                    fn(cfg, r, hawk)
+            for _ in range(3):
+                g.replay()
+            stream.synchronize()
+            a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            n = max(3, min(200, K_steps // n_rep + 1))
+            a0.record(stream)
+            for _ in range(n):
+                g.replay()
+            a1.record(stream)
+            stream.synchronize()
+            kernels[name] = a0.elapsed_time(a1) * 1e3 / (n * n_rep)   # us per launch
+    rej = sum(int((r.accept_len < cfg.K).sum().item()) for r in reps) / n_rep
+    mean_len = float(sum(float(r.accept_len.float().mean().item()) for r in reps) / n_rep)
+    q_rows = sum(int(r.accept_len.clamp(max=cfg.K - 1).add(1).sum().item()) for r in reps) / n_rep
+    stage = {
+        "attn": {"us": kernels["attn"], "GB/s": attn_bytes(cfg) / kernels["attn"] / 1e3,
+                 "frac_hbm": attn_bytes(cfg) / kernels["attn"] / 1e3 / peaks["hbm_gbs"]},
+        "head": {"us": kernels["head"], "GB/s": head_bytes(cfg) / kernels["head"] / 1e3,
+                 "frac_hbm": head_bytes(cfg) / kernels["head"] / 1e3 / peaks["hbm_gbs"],
+                 "TFLOP/s": head_flops(cfg) / kernels["head"] / 1e6,
+                 "frac_tensor": head_flops(cfg) / kernels["head"] / 1e6 / peaks["bf16_tflops"]},
+        "accept": {"us": kernels["accept"], "GB/s": accept_bytes(cfg, cfg.B * cfg.K) / kernels["accept"] / 1e3,
+                   "frac_hbm": accept_bytes(cfg, cfg.B * cfg.K) / kernels["accept"] / 1e3 / peaks["hbm_gbs"],
+                   "bytes_counted": "both logit rows of every position + one q row per position"},
+        "mean_accept_len": mean_len, "sequences_with_rejection": rej, "q_rows_on_chain": q_rows,
+    }
+
+    # ---- end to end through hawk_verify_step_host: pinned host inputs, copies inside the timed region
+    e2e = None
+    if not args.no_e2e:
+        e2e = bench_e2e(cfg, reps, stream, torch, hawk, binding, world, dist, min(K_steps, 2000), W)
+
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K_steps, "warmup": W,
+        "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16 (attention, head operands) / f32 (accumulation, logits, accept)", "data": "synthetic",
+        "config": {"workload": workload_name(cfg, cid), "positions_per_step_per_gpu": positions,
+                   "l2": f"inputs rotate over {n_rep} replicas ({n_rep * first.bytes() / 1e6:.0f} MB > 3x L2)",
+                   "launch": "one CUDA graph replay per step (3 C-ABI calls captured)",
+                   "parallelism": f"{world} independent replicas, sequences sharded, no collective"},
+        "clocks": sampler.summary(), "e2e": e2e, "gpu_launches": launches_per_step * K_steps,
+        "roofline": roofline, "kernels": stage, "dev_status": status,
+    }
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        _, t1, _ = oracle_sample(cfg, wl.seed_for(cid), 1)
+        reps_cpu = max(1, min(50, int(12.0 / max(t1, 1e-3))))      # about 10-15 s of CPU work
+        v, dt, cores = oracle_sample(cfg, wl.seed_for(cid), reps_cpu)
+        line["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle",
+                                "sample": f"{reps_cpu} full steps of the workload ({dt:.1f} s)"}
+    if rank == 0:
+        print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def bench_e2e(cfg, reps, stream, torch, hawk, binding, world, dist, steps, warmup):
+    """Steps through hawk_verify_step_host with pinned host inputs; returns the e2e object."""
+    import ctypes
+    n_rep = len(reps)
+    args_list, keep = [], []
+    for r in reps:
+        host = {k: getattr(r, k).cpu().pin_memory() for k in ("q", "x", "q_probs", "draft", "u_accept", "u_resample")}
+        h_len = torch.empty(cfg.B, dtype=torch.int32).pin_memory()
+        h_tok = torch.empty(cfg.B, dtype=torch.int32).pin_memory()
+        a = binding.StepHostArgs()
+        a.B, a.K, a.H, a.H_kv, a.D, a.L_cap = cfg.B, cfg.K, cfg.H, cfg.H_kv, cfg.D, cfg.L_cap
+        a.max_prefix_len, a.V, a.v_begin, a.v_end, a.top_k = cfg.L, cfg.V, cfg.v_begin, cfg.v_end, cfg.top_k
+        a.sm_scale, a.cfg_scale, a.temperature = r.sm_scale, cfg.cfg_scale, cfg.temperature
+        a.h_q, a.h_x, a.h_q_probs = host["q"].data_ptr(), host["x"].data_ptr(), host["q_probs"].data_ptr()
+        a.h_draft, a.h_u_accept, a.h_u_resample = (host["draft"].data_ptr(), host["u_accept"].data_ptr(),
+                                                   host["u_resample"].data_ptr())
+        a.h_accept_len, a.h_out_token = h_len.data_ptr(), h_tok.data_ptr()
+        a.d_k_cache, a.d_v_cache, a.d_prefix_len, a.d_w = (r.k_cache.data_ptr(), r.v_cache.data_ptr(),
+                                                           r.prefix_len.data_ptr(), r.w.data_ptr())
+        a.d_q, a.d_x, a.d_q_probs, a.d_draft = r.q.data_ptr(), r.x.data_ptr(), r.q_probs.data_ptr(), r.draft.data_ptr()
+        a.d_u_accept, a.d_u_resample = r.u_accept.data_ptr(), r.u_resample.data_ptr()
+        a.d_attn_out, a.d_logits = r.attn_out.data_ptr(), r.logits.data_ptr()
+        a.d_accept_len, a.d_out_token = r.accept_len.data_ptr(), r.out_token.data_ptr()
+        a.d_attn_workspace, a.attn_workspace_bytes = r.attn_ws.data_ptr(), r.attn_ws.numel()
+        a.d_accept_workspace, a.accept_workspace_bytes = r.acc_ws.data_ptr(), r.acc_ws.numel()
+        a.d_status = r.status.data_ptr()
+        args_list.append(a)
+        keep.append((host, h_len, h_tok))
+    h2d = sum(t.numel() * t.element_size() for t in keep[0][0].values())
+    d2h = 2 * cfg.B * 4
+    start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    with torch.cuda.stream(stream):
+        for i in range(warmup):
+            hawk.verify_step_host(args_list[i % n_rep])
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+        start.record(stream)
+        for i in range(steps):
+            hawk.verify_step_host(args_list[i % n_rep])
+        stop.record(stream)
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+    ms = start.elapsed_time(stop)
+    if dist is not None:
+        t = torch.tensor([ms], device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+    return {"value": cfg.B * cfg.K * world / (ms / steps * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+            "d2h_bytes_per_step": d2h, "ms_per_step": ms / steps, "steps": steps,
+            "api": "hawk_verify_step_host (pinned host inputs -> device, 3 kernels, results -> host)"}
+
+
+if __name__ == "__main__":
+    main()

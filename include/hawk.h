@@ -99,7 +99,7 @@ hawk_status hawk_verify_attn(const void *q, const void *k_cache, const void *v_c
  *   x       bf16 [M][hidden]   one row per (stream, draft position): M = 2*B*K
  *   w       bf16 [V][hidden]   one row per token id
  *   logits  fp32 [M][V]
- * Supported: hidden a multiple of 64; V a multiple of 4 and logits 16-byte aligned.
+ * Supported: hidden a multiple of 64 (and >= 64).
  * Errors: NULL, SHAPE (negative sizes, range outside [0, V]), ALIGN, UNSUPPORTED, CUDA.
  * M == 0 or an empty range returns HAWK_OK without a launch.
  * ---------------------------------------------------------------------------------------------- */
@@ -151,6 +151,54 @@ hawk_status hawk_cfg_accept(const float *logits, const float *q_probs, const int
                             int has_bonus_row, int32_t *accept_len, int32_t *out_token,
                             float *p_debug, void *workspace, size_t workspace_bytes,
                             int32_t *dev_status, hawk_stream_t stream);
+
+/* ------------------------------------------------------------------------------------------------
+ * hawk_verify_step_host - one whole verify step with the per-step inputs in HOST memory.
+ *
+ * Runs, on `stream`: host->device copies of the step's inputs into the caller's device staging,
+ * hawk_verify_attn, hawk_head_proj, hawk_cfg_accept (contracts above, no bonus row), and
+ * device->host copies of accept_len and out_token.  The attention output and the head input are
+ * separate tensors: the layers between them (output projection, MLP, norm) are not part of this
+ * library, so x is an input of the step like q.  The call returns once everything is queued; the
+ * results are valid after the stream has been synchronised.  Use pinned host memory for the copies
+ * to be asynchronous.  The KV cache, the head weight and the prefix lengths are resident device
+ * state; all d_* staging and workspaces are device memory owned by the caller.
+ * Errors: as the three stage calls, plus HAWK_ERR_CUDA if a copy is refused.
+ * ---------------------------------------------------------------------------------------------- */
+typedef struct {
+    /* sizes and sampling parameters */
+    int B, K, H, H_kv, D, L_cap, max_prefix_len, V, v_begin, v_end, top_k;
+    float sm_scale, cfg_scale, temperature;
+    /* per-step inputs, host */
+    const void *h_q;            /* bf16 [2B][K][H][D]      */
+    const void *h_x;            /* bf16 [2B*K][H*D]        */
+    const float *h_q_probs;     /* fp32 [B][K][V]          */
+    const int32_t *h_draft;     /* [B][K]                  */
+    const float *h_u_accept;    /* [B][K]                  */
+    const float *h_u_resample;  /* [B][K+1]                */
+    /* per-step results, host */
+    int32_t *h_accept_len;      /* [B] */
+    int32_t *h_out_token;       /* [B] */
+    /* resident device state */
+    const void *d_k_cache, *d_v_cache;   /* bf16 [2B][H_kv][L_cap][D] */
+    const int32_t *d_prefix_len;         /* [2B] */
+    const void *d_w;                     /* bf16 [V][H*D] */
+    /* device staging for the inputs, intermediates and results (same shapes as above) */
+    void *d_q, *d_x;
+    float *d_q_probs;
+    int32_t *d_draft;
+    float *d_u_accept, *d_u_resample;
+    void *d_attn_out;           /* bf16 [2B][K][H*D] */
+    float *d_logits;            /* fp32 [2B*K][V]    */
+    int32_t *d_accept_len, *d_out_token;
+    void *d_attn_workspace;
+    size_t attn_workspace_bytes;
+    void *d_accept_workspace;
+    size_t accept_workspace_bytes;
+    int32_t *d_status;          /* optional */
+} hawk_step_host_args;
+
+hawk_status hawk_verify_step_host(const hawk_step_host_args *args, hawk_stream_t stream);
 
 #ifdef __cplusplus
 }

@@ -11,6 +11,7 @@ _BINDING_NAMES = (
     "load_library", "library_path", "HawkError", "status_string", "version",
     "verify_attn", "verify_attn_workspace_bytes", "head_proj",
     "cfg_accept", "cfg_accept_workspace_bytes",
+    "verify_step_host", "StepHostArgs",
 )
 
 

@@ -23,7 +23,26 @@ EXPORTS = (
     "hawk_verify_attn_workspace_bytes", "hawk_verify_attn",
     "hawk_head_proj",
     "hawk_cfg_accept_workspace_bytes", "hawk_cfg_accept",
+    "hawk_verify_step_host",
 )
+
+
+def _step_fields():
+    vp, i32, f32, sz = ctypes.c_void_p, ctypes.c_int, ctypes.c_float, ctypes.c_size_t
+    ints = ("B", "K", "H", "H_kv", "D", "L_cap", "max_prefix_len", "V", "v_begin", "v_end", "top_k")
+    floats = ("sm_scale", "cfg_scale", "temperature")
+    ptrs = ("h_q", "h_x", "h_q_probs", "h_draft", "h_u_accept", "h_u_resample", "h_accept_len", "h_out_token",
+            "d_k_cache", "d_v_cache", "d_prefix_len", "d_w",
+            "d_q", "d_x", "d_q_probs", "d_draft", "d_u_accept", "d_u_resample",
+            "d_attn_out", "d_logits", "d_accept_len", "d_out_token", "d_attn_workspace")
+    return ([(n, i32) for n in ints] + [(n, f32) for n in floats] + [(n, vp) for n in ptrs]
+            + [("attn_workspace_bytes", sz), ("d_accept_workspace", vp), ("accept_workspace_bytes", sz),
+               ("d_status", vp)])
+
+
+class StepHostArgs(ctypes.Structure):
+    """Mirror of hawk_step_host_args (include/hawk.h)."""
+    _fields_ = _step_fields()
 
 
 class HawkError(RuntimeError):
@@ -62,6 +81,8 @@ def load_library() -> ctypes.CDLL:
     lib.hawk_cfg_accept.restype = i32
     lib.hawk_cfg_accept.argtypes = [vp, vp, vp, vp, vp, i32, i32, i32, i32, i32, f32, f32, i32, i32,
                                     vp, vp, vp, vp, sz, vp, vp]
+    lib.hawk_verify_step_host.restype = i32
+    lib.hawk_verify_step_host.argtypes = [ctypes.POINTER(StepHostArgs), vp]
     _lib = lib
     return lib
 
@@ -180,3 +201,10 @@ def cfg_accept(logits: torch.Tensor, q_probs: torch.Tensor, draft: torch.Tensor,
     if rc != 0:
         raise HawkError(rc, "hawk_cfg_accept")
     return accept_len, out_token
+
+
+def verify_step_host(args: StepHostArgs) -> None:
+    """Queues one whole verify step (copies in, three kernels, copies out) on the current stream."""
+    rc = load_library().hawk_verify_step_host(ctypes.byref(args), _stream())
+    if rc != 0:
+        raise HawkError(rc, "hawk_verify_step_host")
