@@ -75,7 +75,7 @@ def accept_bytes(cfg, q_rows_read: int) -> int:
 class ClockSampler:
     """Samples SM clock and throttle reasons through NVML while the timed region runs."""
 
-    def __init__(self, index: int, uuid: str = "", period_s: float = 0.05):
+    def __init__(self, index: int, uuid: str = "", period_s: float = 0.01):
         self.index, self.period = index, period_s
         self.samples, self.reasons, self.max_mhz = [], set(), None
         self._stop = threading.Event()
@@ -459,7 +459,7 @@ def main():
     }
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         _, t1, _ = oracle_sample(cfg, wl.seed_for(cid), 1)
-        reps_cpu = max(1, min(50, int(12.0 / max(t1, 1e-3))))      # about 10-15 s of CPU work
+        reps_cpu = max(1, min(500, int(12.0 / max(t1, 1e-3))))     # about 10-15 s of CPU work
         v, dt, cores = oracle_sample(cfg, wl.seed_for(cid), reps_cpu)
         line["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle",
                                 "sample": f"{reps_cpu} full steps of the workload ({dt:.1f} s)"}

@@ -1,0 +1,130 @@
+"""The C-ABI library loads, exports every function include/hawk.h declares, and its host-side
+argument checks return the documented codes.  Nothing here launches a kernel: every call below is
+rejected (or is a no-op) before the library touches a device."""
+import ctypes
+import re
+from pathlib import Path
+
+import pytest
+
+from paper_2510_25739_b200 import binding, build
+
+HEADER = Path(__file__).resolve().parent.parent / "include" / "hawk.h"
+OK, E_NULL, E_SHAPE, E_ALIGN, E_UNSUP, E_WS, E_PARAM, E_CUDA = range(8)
+
+
+@pytest.fixture(scope="module")
+def lib():
+    build.build()
+    return binding.load_library()
+
+
+def _declared_functions():
+    text = re.sub(r"/\*.*?\*/", "", HEADER.read_text(), flags=re.S)
+    return sorted(set(re.findall(r"\b(hawk_[a-z_]+)\s*\(", text)))
+
+
+def test_every_declared_function_is_exported(lib):
+    names = _declared_functions()
+    assert {"hawk_verify_attn", "hawk_head_proj", "hawk_cfg_accept"} <= set(names)
+    for n in names:
+        assert hasattr(lib, n), f"{n} is declared in hawk.h but not exported"
+    assert set(binding.EXPORTS) == set(names)
+
+
+def test_version_and_status_strings(lib):
+    assert lib.hawk_version() >= 100
+    seen = {lib.hawk_status_string(c).decode() for c in range(8)}
+    assert len(seen) == 8 and "ok" in seen
+    assert lib.hawk_status_string(99).decode() == "unknown status"
+
+
+def test_step_struct_matches_the_header():
+    text = HEADER.read_text()
+    body = text[text.index("typedef struct {"):text.index("} hawk_step_host_args;")]
+    body = re.sub(r"/\*.*?\*/", "", body, flags=re.S)
+    names = []
+    for decl in body.split(";"):
+        decl = decl.replace("typedef struct {", "").strip()
+        if not decl:
+            continue
+        parts = re.sub(r"^(const\s+)?(void|float|int32_t|int|size_t)\b", "", decl).split(",")
+        names += [p.replace("*", "").strip() for p in parts]
+    assert names == [f[0] for f in binding.StepHostArgs._fields_]
+
+
+def test_workspace_queries(lib):
+    # invalid shapes report 0; a split launch needs (D + 2) floats per (row, split)
+    assert lib.hawk_verify_attn_workspace_bytes(0, 4, 16, 16, 64, 128) == 0
+    assert lib.hawk_verify_attn_workspace_bytes(2, 4, 16, 16, 96, 128) == 0
+    need = lib.hawk_verify_attn_workspace_bytes(16, 5, 20, 20, 64, 1144)
+    assert need % (16 * 20 * 5 * 66 * 4) == 0
+    assert lib.hawk_cfg_accept_workspace_bytes(8, 5, 16384) >= 8 * 5 * 4
+    assert lib.hawk_cfg_accept_workspace_bytes(0, 5, 16384) == 0
+
+
+def test_attn_argument_checks(lib):
+    p = ctypes.c_void_p(0x1000)          # never dereferenced: every call below fails a host check first
+    odd = ctypes.c_void_p(0x1004)
+    f = lib.hawk_verify_attn
+    args = dict(S=2, K=4, H=16, H_kv=16, D=64, L_cap=132, mpl=128, scale=0.125)
+
+    def call(q=p, k=p, v=p, pl=p, out=p, ws=None, wsb=0, **kw):
+        a = {**args, **kw}
+        return f(q, k, v, pl, out, a["S"], a["K"], a["H"], a["H_kv"], a["D"], a["L_cap"], a["mpl"], a["scale"],
+                 ws, wsb, None, None)
+
+    assert call(S=0) == OK
+    assert call(S=-1) == E_SHAPE
+    assert call(q=None) == E_NULL
+    assert call(out=None) == E_NULL
+    assert call(K=0) == E_UNSUP and call(K=17) == E_UNSUP
+    assert call(D=96) == E_UNSUP
+    assert call(H=16, H_kv=3) == E_UNSUP
+    assert call(mpl=129) == E_SHAPE                      # prefix + K exceeds the cache capacity
+    assert call(scale=0.0) == E_PARAM and call(scale=float("nan")) == E_PARAM
+    assert call(scale=float("inf")) == E_PARAM
+    assert call(k=odd) == E_ALIGN
+    assert call(S=2 ** 20, L_cap=2 ** 12, mpl=100) == E_UNSUP   # row index would overflow 31 bits
+
+
+def test_head_argument_checks(lib):
+    p, odd = ctypes.c_void_p(0x1000), ctypes.c_void_p(0x1008)
+    f = lib.hawk_head_proj
+    assert f(p, p, p, 0, 1024, 16384, 0, 16384, None, None) == OK
+    assert f(p, p, p, 8, 1024, 16384, 5, 5, None, None) == OK       # empty range
+    assert f(p, p, p, -1, 1024, 16384, 0, 16384, None, None) == E_SHAPE
+    assert f(p, p, p, 8, 1024, 16384, 0, 16385, None, None) == E_SHAPE
+    assert f(p, p, p, 8, 1024, 16384, 9, 8, None, None) == E_SHAPE
+    assert f(None, p, p, 8, 1024, 16384, 0, 16384, None, None) == E_NULL
+    assert f(p, p, p, 8, 1000, 16384, 0, 16384, None, None) == E_UNSUP   # hidden not a multiple of 64
+    assert f(p, odd, p, 8, 1024, 16384, 0, 16384, None, None) == E_ALIGN
+
+
+def test_accept_argument_checks(lib):
+    p, odd = ctypes.c_void_p(0x1000), ctypes.c_void_p(0x1004)
+    f = lib.hawk_cfg_accept
+
+    def call(lg=p, q=p, d=p, ua=p, ur=p, B=2, K=4, V=1024, vb=0, ve=1024, s=3.0, T=1.0, k=100, al=p, tok=p,
+             ws=p, wsb=1 << 20):
+        return f(lg, q, d, ua, ur, B, K, V, vb, ve, s, T, k, 0, al, tok, None, ws, wsb, None, None)
+
+    assert call(B=0) == OK
+    assert call(B=-1) == E_SHAPE
+    assert call(lg=None) == E_NULL and call(tok=None) == E_NULL
+    assert call(vb=10, ve=10) == E_SHAPE and call(ve=2000) == E_SHAPE
+    assert call(K=0) == E_UNSUP and call(K=17) == E_UNSUP
+    assert call(V=40000, ve=40000) == E_UNSUP            # more valid ids than one block holds
+    assert call(T=0.0) == E_PARAM and call(T=-1.0) == E_PARAM and call(T=float("nan")) == E_PARAM
+    assert call(s=float("inf")) == E_PARAM
+    assert call(q=odd) == E_ALIGN
+    assert call(ws=None) == E_WS and call(wsb=4) == E_WS
+
+
+def test_step_host_argument_checks(lib):
+    assert lib.hawk_verify_step_host(None, None) == E_NULL
+    a = binding.StepHostArgs()
+    a.B = 0
+    assert lib.hawk_verify_step_host(ctypes.byref(a), None) == OK
+    a.B, a.K, a.H, a.D, a.V = 1, 4, 16, 64, 16384
+    assert lib.hawk_verify_step_host(ctypes.byref(a), None) == E_NULL     # no buffers given
