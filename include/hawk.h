@@ -153,6 +153,36 @@ hawk_status hawk_cfg_accept(const float *logits, const float *q_probs, const int
                             int32_t *dev_status, hawk_stream_t stream);
 
 /* ------------------------------------------------------------------------------------------------
+ * hawk_cfg_accept_noalloc - hawk_cfg_accept without a caller-provided workspace.
+ *
+ * The paper has no counterpart of this call; it exists for the way the library gets embedded.
+ * Some callers cannot obtain device memory at the moment they need a verdict: a decode loop running
+ * inside a serving engine whose memory manager took the whole device at start-up (a fresh
+ * allocation there fails, or stalls every stream while the driver serves it), or a plug-in that is
+ * handed its input and output buffers by a host application and owns nothing else.  For them the
+ * per-row verdicts go to a fixed 64 KiB array that is part of the library's device image; every GPU
+ * that loads the library carries that array until the process exits.
+ *
+ * Same operation, arguments and results as hawk_cfg_accept, minus p_debug, workspace and
+ * workspace_bytes.  Limit: B * (K + 1) <= hawk_cfg_accept_noalloc_max_rows() (16384); a larger step
+ * returns HAWK_ERR_WORKSPACE and launches nothing.  The call allocates and frees nothing.
+ *
+ * The first call on each device looks up the array's device address (one runtime query, made with
+ * that device current); make that first call outside any stream capture.
+ * All calls on a device share the one array, and it keeps the previous call's contents.  Nothing in
+ * it has to start at zero (each row's slot is rewritten before it is read), but two calls whose
+ * kernels overlap on the GPU - different streams without an ordering between them - race on it:
+ * order such calls, or give the concurrent ones their own workspace through hawk_cfg_accept.
+ * ---------------------------------------------------------------------------------------------- */
+size_t hawk_cfg_accept_noalloc_max_rows(void);
+
+hawk_status hawk_cfg_accept_noalloc(const float *logits, const float *q_probs, const int32_t *draft,
+                                    const float *u_accept, const float *u_resample, int B, int K, int V,
+                                    int v_begin, int v_end, float cfg_scale, float temperature,
+                                    int top_k, int has_bonus_row, int32_t *accept_len,
+                                    int32_t *out_token, int32_t *dev_status, hawk_stream_t stream);
+
+/* ------------------------------------------------------------------------------------------------
  * hawk_verify_step_host - one whole verify step with the per-step inputs in HOST memory.
  *
  * Runs, on `stream`: host->device copies of the step's inputs into the caller's device staging,

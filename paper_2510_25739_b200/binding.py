@@ -24,6 +24,7 @@ EXPORTS = (
     "hawk_head_proj",
     "hawk_cfg_accept_workspace_bytes", "hawk_cfg_accept",
     "hawk_verify_step_host",
+    "hawk_cfg_accept_noalloc_max_rows", "hawk_cfg_accept_noalloc",
 )
 
 
@@ -81,6 +82,11 @@ def load_library() -> ctypes.CDLL:
     lib.hawk_cfg_accept.restype = i32
     lib.hawk_cfg_accept.argtypes = [vp, vp, vp, vp, vp, i32, i32, i32, i32, i32, f32, f32, i32, i32,
                                     vp, vp, vp, vp, sz, vp, vp]
+    lib.hawk_cfg_accept_noalloc_max_rows.restype = sz
+    lib.hawk_cfg_accept_noalloc_max_rows.argtypes = []
+    lib.hawk_cfg_accept_noalloc.restype = i32
+    lib.hawk_cfg_accept_noalloc.argtypes = [vp, vp, vp, vp, vp, i32, i32, i32, i32, i32, f32, f32, i32, i32,
+                                            vp, vp, vp, vp]
     lib.hawk_verify_step_host.restype = i32
     lib.hawk_verify_step_host.argtypes = [ctypes.POINTER(StepHostArgs), vp]
     _lib = lib
@@ -200,6 +206,36 @@ def cfg_accept(logits: torch.Tensor, q_probs: torch.Tensor, draft: torch.Tensor,
                              _ptr(workspace), ws_bytes, _ptr(dev_status), _stream())
     if rc != 0:
         raise HawkError(rc, "hawk_cfg_accept")
+    return accept_len, out_token
+
+
+def cfg_accept_noalloc_max_rows() -> int:
+    return int(load_library().hawk_cfg_accept_noalloc_max_rows())
+
+
+def cfg_accept_noalloc(logits: torch.Tensor, q_probs: torch.Tensor, draft: torch.Tensor, u_accept: torch.Tensor,
+                       u_resample: torch.Tensor, v_begin: int, v_end: int, cfg_scale: float, temperature: float,
+                       top_k: int, accept_len: torch.Tensor, out_token: torch.Tensor, has_bonus_row: bool = False,
+                       dev_status: Optional[torch.Tensor] = None):
+    """cfg_accept for callers that cannot lend a workspace: the verdict scratch is the library's built-in
+    array.  Nothing is allocated here either, so both result tensors ([B] int32) must be passed in.
+    Steps with B * (K + 1) above cfg_accept_noalloc_max_rows() are refused (HawkError, workspace)."""
+    lib = load_library()
+    B, K, V = q_probs.shape
+    rows = K + (1 if has_bonus_row else 0)
+    _check(logits, torch.float32, "logits", (2 * B, rows, V))
+    _check(q_probs, torch.float32, "q_probs")
+    _check(draft, torch.int32, "draft", (B, K))
+    _check(u_accept, torch.float32, "u_accept", (B, K))
+    _check(u_resample, torch.float32, "u_resample", (B, K + 1))
+    _check(accept_len, torch.int32, "accept_len", (B,))
+    _check(out_token, torch.int32, "out_token", (B,))
+    rc = lib.hawk_cfg_accept_noalloc(_ptr(logits), _ptr(q_probs), _ptr(draft), _ptr(u_accept), _ptr(u_resample),
+                                     B, K, V, int(v_begin), int(v_end), float(cfg_scale), float(temperature),
+                                     int(top_k), int(bool(has_bonus_row)), _ptr(accept_len), _ptr(out_token),
+                                     _ptr(dev_status), _stream())
+    if rc != 0:
+        raise HawkError(rc, "hawk_cfg_accept_noalloc")
     return accept_len, out_token
 
 

@@ -11,6 +11,8 @@
 // (speculative sampling, Sec. 3; chain verification and residual update, Sec. 4.2).
 #include <math_constants.h>
 
+#include <mutex>
+
 #include "hawk_common.cuh"
 
 namespace {
@@ -556,4 +558,57 @@ extern "C" hawk_status hawk_cfg_accept(const float *logits, const float *q_probs
     if (err != cudaSuccess) return HAWK_ERR_CUDA;
     accept_finalize_kernel<<<(B + 127) / 128, 128, 0, st>>>(P.row_out, B, K, P.rows, accept_len, out_token);
     return cudaGetLastError() == cudaSuccess ? HAWK_OK : HAWK_ERR_CUDA;
+}
+
+// ------------------------------------------------------------------------------------------------
+// hawk_cfg_accept_noalloc: the same verification for callers that have no device memory to lend
+// as a workspace.  The per-row verdicts go to a fixed array that lives in the library's own
+// device image instead.
+namespace {
+
+constexpr int kBuiltinRows = 16384;  // verdict slots: B * (K + 1) must not exceed this (64 KiB)
+static __device__ __align__(256) int32_t g_builtin_row_out[kBuiltinRows];
+
+constexpr int kMaxDevices = 64;
+std::mutex g_builtin_mutex;
+void *g_builtin_addr[kMaxDevices];  // device address of the array, per device, once looked up
+
+// The array's name is only a host-side handle; kernels need its device address, which differs per
+// device.  Looked up once per device, with that device current.
+hawk_status builtin_scratch(void **ptr)
+{
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return HAWK_ERR_CUDA;
+    std::lock_guard<std::mutex> lock(g_builtin_mutex);
+    if (!g_builtin_addr[dev]) {
+        void *p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_builtin_row_out) != cudaSuccess || !p) return HAWK_ERR_CUDA;
+        g_builtin_addr[dev] = p;
+    }
+    *ptr = g_builtin_addr[dev];
+    return HAWK_OK;
+}
+
+}  // namespace
+
+extern "C" size_t hawk_cfg_accept_noalloc_max_rows(void) { return kBuiltinRows; }
+
+extern "C" hawk_status hawk_cfg_accept_noalloc(const float *logits, const float *q_probs, const int32_t *draft,
+                                               const float *u_accept, const float *u_resample, int B, int K, int V,
+                                               int v_begin, int v_end, float cfg_scale, float temperature,
+                                               int top_k, int has_bonus_row, int32_t *accept_len,
+                                               int32_t *out_token, int32_t *dev_status, hawk_stream_t stream)
+{
+    if (B < 0 || K < 0 || V < 0) return HAWK_ERR_SHAPE;
+    if (B == 0) return HAWK_OK;
+    if (K < 1 || K > 16) return HAWK_ERR_UNSUPPORTED;
+    if (static_cast<long long>(B) * (K + 1) > kBuiltinRows) return HAWK_ERR_WORKSPACE;  // beyond the built-in array
+    void *scratch = nullptr;
+    const hawk_status rc = builtin_scratch(&scratch);
+    if (rc != HAWK_OK) return rc;
+    // Every row of the step writes its own slot before the per-sequence pass reads it, so the array
+    // needs no clearing even though it still holds the previous call's verdicts.
+    return hawk_cfg_accept(logits, q_probs, draft, u_accept, u_resample, B, K, V, v_begin, v_end, cfg_scale,
+                           temperature, top_k, has_bonus_row, accept_len, out_token, nullptr, scratch,
+                           sizeof(int32_t) * kBuiltinRows, dev_status, stream);
 }
