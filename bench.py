@@ -287,6 +287,8 @@ def main():
     ap.add_argument("--impl", default="hawk", choices=["hawk", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--graph-events", action="store_true",
+                    help="also record events around the attention call inside the step graphs (perturbs the step)")
     args = ap.parse_args()
     cid = args.config
     cfg = wl.config(cid)
@@ -322,7 +324,7 @@ def main():
 
     # ---- one CUDA graph per replica: [ev0] attn [ev1] head accept
     graphs, evs = [], []
-    external_events = True
+    external_events = bool(args.graph_events)
     with torch.cuda.stream(stream):
         for r in reps:                       # warm the kernels (function attributes are set on first use)
             run_attn(cfg, r, hawk); run_head(cfg, r, hawk); run_accept(cfg, r, hawk)
@@ -385,7 +387,7 @@ def main():
         except Exception:
             attn_ms = []
     if not attn_ms:
-        timing_mode = "attention-only loop (graph event nodes unavailable)"
+        timing_mode = "attention-only launches back to back on the bench stream, replicas rotating (L2-cold)"
         with torch.cuda.stream(stream):
             a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             n = max(50, min(K_steps, 500))

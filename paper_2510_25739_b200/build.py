@@ -41,6 +41,7 @@ def build(force: bool = False, verbose: bool = False) -> Path:
            "-cudart", "static", "-o", str(tmp)]
     if verbose:
         cmd += ["-Xptxas", "-v"]
+    cmd += os.environ.get("HAWK_NVCC_FLAGS", "").split()   # e.g. -DHAWK_ATTN_WARPS=4 -DHAWK_ATTN_STAGE_KB=16
     cmd += [str(CSRC / s) for s in SOURCES]
     res = subprocess.run(cmd, capture_output=True, text=True)
     if res.returncode != 0:

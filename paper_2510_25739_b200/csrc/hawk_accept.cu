@@ -169,6 +169,8 @@ __global__ void __launch_bounds__(NT) accept_rows_kernel(const AcceptParams P)
     __shared__ float s_tau, s_px;
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    hawk::allow_dependent_launch();
+    hawk::grid_dependency_wait();
     const int row = blockIdx.x;  // position-major: all rows of position 0 first
     const int i = row / P.B, b = row - i * P.B;
     const bool bonus = (i == P.K);
@@ -468,6 +470,8 @@ __global__ void __launch_bounds__(NT) accept_rows_kernel(const AcceptParams P)
 __global__ void accept_finalize_kernel(const int32_t *row_out, int B, int K, int rows, int32_t *accept_len,
                                        int32_t *out_token)
 {
+    hawk::allow_dependent_launch();
+    hawk::grid_dependency_wait();
     const int b = blockIdx.x * blockDim.x + threadIdx.x;
     if (b >= B) return;
     int len = K, tok = -1;
@@ -490,8 +494,7 @@ __global__ void accept_finalize_kernel(const int32_t *row_out, int B, int K, int
 template <int NT, int VPT>
 cudaError_t launch_rows(const AcceptParams &P, int grid, cudaStream_t stream)
 {
-    accept_rows_kernel<NT, VPT><<<grid, NT, 0, stream>>>(P);
-    return cudaGetLastError();
+    return hawk_host::launch_dependent(accept_rows_kernel<NT, VPT>, dim3(grid), dim3(NT), 0, stream, P);
 }
 
 }  // namespace
@@ -556,8 +559,9 @@ extern "C" hawk_status hawk_cfg_accept(const float *logits, const float *q_probs
     else if (n <= 16384) err = launch_rows<512, 8>(P, grid, st);
     else err = launch_rows<1024, 8>(P, grid, st);
     if (err != cudaSuccess) return HAWK_ERR_CUDA;
-    accept_finalize_kernel<<<(B + 127) / 128, 128, 0, st>>>(P.row_out, B, K, P.rows, accept_len, out_token);
-    return cudaGetLastError() == cudaSuccess ? HAWK_OK : HAWK_ERR_CUDA;
+    err = hawk_host::launch_dependent(accept_finalize_kernel, dim3((B + 127) / 128), dim3(128), 0, st,
+                                      static_cast<const int32_t *>(P.row_out), B, K, P.rows, accept_len, out_token);
+    return err == cudaSuccess ? HAWK_OK : HAWK_ERR_CUDA;
 }
 
 // ------------------------------------------------------------------------------------------------

@@ -1,16 +1,23 @@
 // hawk_verify_attn: block-causal attention of the K draft queries of every guidance stream against
 // the cached keys/values (the target model's parallel verification pass, Sec. 3).
 //
-// The kernel is bound by reading the KV cache once from HBM.  Each thread block owns one
-// (stream, kv head, query-head chunk, key split) item and streams its keys through shared memory:
-//   - one producer warp issues TMA tile loads (128-byte swizzle) into a ring of stages guarded by
-//     full/empty mbarriers;
-//   - four consumer warps each take 16 keys of every 64-key tile, compute Q.K^T and P.V with
-//     warp-level bf16 MMAs (queries padded to the 16-row operand; the tensor pipe is only an ALU
-//     offload here) and keep a running max/sum softmax in registers with quad shuffles;
-//   - the four partial results are merged through shared memory and either written as bf16 or, when
-//     the keys of an item are split over several blocks, stored as fp32 partials that a small
-//     second kernel merges.
+// The kernel is bound by reading the KV cache once from HBM, so it is organised around keeping
+// that stream of bytes flowing without a gap:
+//   - The work is the flat list of KV tiles (item-major; an item is one (stream, kv head, chunk of
+//     <= 16 query rows), a tile is kTileKeys consecutive keys).  The list is cut into equal contiguous
+//     shares, one per warp of a persistent grid (one block per SM), so every warp reads the same
+//     number of bytes whatever the shape of the batch and no wave of blocks is ever partly empty.
+//   - Each warp is its own pipeline: lane 0 issues TMA tile loads (128-byte swizzle) into the warp's
+//     private ring of stages and re-arms a stage right after the warp has consumed it; there is no
+//     block-wide synchronisation after start-up.
+//   - Per tile the warp computes the transposed products S^T = K.Q^T and O^T = V^T.P^T with warp-level
+//     bf16 MMAs: the keys (and the head dimension) sit on the 16-row operand, the handful of draft
+//     queries on the 8-column operand, so a block of K <= 8 drafts wastes no tensor work and the
+//     per-key softmax work is a quarter of the query-major form.  The tensor pipe is only an ALU
+//     offload here; running max/sum softmax stays in registers (one max reduction per tile).
+//   - A share that holds all tiles of an item writes bf16 output straight from registers.  A share
+//     that holds only part of an item stores an fp32 partial (o, max, sum) in the workspace, and a
+//     small second kernel merges the partials of every item that was cut.
 #include <math_constants.h>
 
 #include "hawk_common.cuh"
@@ -19,387 +26,576 @@ namespace {
 
 using namespace hawk;
 
-constexpr int kConsumerWarps = 4;
-constexpr int kKeysPerWarp = 16;
-constexpr int kTileKeys = kConsumerWarps * kKeysPerWarp;  // 64 keys per stage
-constexpr int kThreads = (kConsumerWarps + 1) * 32;
+#ifndef HAWK_ATTN_WARPS
+#define HAWK_ATTN_WARPS 8
+#endif
+#ifndef HAWK_ATTN_STAGE_KB
+#define HAWK_ATTN_STAGE_KB 8
+#endif
+constexpr int kWarps = HAWK_ATTN_WARPS;  // independent pipelines per block
+constexpr int kThreads = kWarps * 32;
+constexpr int kStages = 3;               // ring depth of one warp
+constexpr int kStageBytes = HAWK_ATTN_STAGE_KB * 1024;  // K and V tile of one stage
+constexpr int kPlanSms = 148;           // launch shape is planned for the B200's 148 SMs
 
 template <int D>
 struct AttnCfg {
-    static constexpr int kHalves = D / 64;                        // 64-column (128-byte) sub-tiles
-    static constexpr int kSubTileBytes = kTileKeys * 128;         // one [64 keys][64 cols] sub-tile
-    static constexpr int kStageBytes = 2 * kHalves * kSubTileBytes;  // K and V
-    static constexpr int kStages = D == 64 ? 4 : 3;
-    static constexpr int kMergeFloats = kConsumerWarps * 16 * (D + 2);  // aliases the stage ring after the loop
-    static_assert(kMergeFloats * sizeof(float) <= static_cast<size_t>(kStages) * kStageBytes, "merge must fit");
+    static constexpr int kHalves = D / 64;                       // 64-column (128-byte) sub-tiles
+    static constexpr int kTileKeys = kStageBytes / (4 * D);      // keys per stage (K row + V row = 4*D bytes)
+    static_assert(kTileKeys % 16 == 0 && kTileKeys >= 16, "a tile is a whole number of 16-key MMA blocks");
+    static constexpr int kSubTileBytes = kTileKeys * 128;        // one [keys][64 cols] sub-tile
+    static_assert(2 * kHalves * kSubTileBytes == kStageBytes, "stage = K tile + V tile");
     static constexpr size_t kSmemBytes =
-        1024 /*align slack*/ + static_cast<size_t>(kStages) * kStageBytes + 2 * kStages * sizeof(uint64_t) + 64;
+        1024 /*align slack*/ + static_cast<size_t>(kWarps) * kStages * kStageBytes + kWarps * kStages * sizeof(uint64_t);
 };
 
 struct AttnParams {
     const __nv_bfloat16 *q;
     const int32_t *prefix_len;
     __nv_bfloat16 *out;
-    float *part_o;   // [S][H][K][nsplit][D]
-    float *part_ml;  // [S][H][K][nsplit][2]
+    float *part;  // [workers][2 slots]{o[16 rows][D], (running max in log2 units, running sum)[16 rows]}
     int S, K, H, H_kv, L_cap;
-    int chunk_heads;  // query heads handled per item (rows = chunk_heads * K <= 16)
-    int chunks;       // items per kv head
-    int nsplit;
-    float scale_log2;  // sm_scale * log2(e)
+    int pl_max;           // largest admissible prefix length: min(L_cap - K, max_prefix_len)
+    int chunk_heads;      // query heads handled per item (rows = chunk_heads * K <= 16)
+    int chunks;           // items per kv head
+    int tiles_per_item;   // tiles of the longest admissible prefix: ceil((max_prefix_len + K) / kTileKeys)
+    int workers;          // warps that own a share of the flat tile list
+    long long total_tiles;  // items * tiles_per_item
+    float scale_log2;     // sm_scale * log2(e)
     int32_t *dev_status;
 };
 
-template <int D>
-__global__ void __launch_bounds__(kThreads) attn_kernel(const __grid_constant__ CUtensorMap map_k,
-                                                        const __grid_constant__ CUtensorMap map_v,
-                                                        const AttnParams P)
+// Flat tile f belongs to worker owner(f); worker g owns [share_begin(g), share_begin(g + 1)).
+__host__ __device__ __forceinline__ long long share_begin(long long g, long long T, int G) { return g * T / G; }
+__host__ __device__ __forceinline__ int owner(long long f, long long T, int G)
+{
+    return static_cast<int>(((f + 1) * G - 1) / T);
+}
+
+// Position in the flat tile list, decoded.
+struct Cursor {
+    long long f;
+    int item, tile;             // tile index inside the item
+    int s, hk, chunk;           // stream, kv head, row chunk
+    int pl;                     // clamped prefix length of the stream
+    int ntiles;                 // tiles that hold visible keys for this stream
+    int row_base;               // first cache row of (s, hk)
+};
+
+template <int TK>
+__device__ __forceinline__ void decode_item(Cursor &c, const AttnParams &P, int &flags)
+{
+    c.item = static_cast<int>(c.f / P.tiles_per_item);
+    c.tile = static_cast<int>(c.f - static_cast<long long>(c.item) * P.tiles_per_item);
+    int it = c.item;
+    c.chunk = it % P.chunks;
+    it /= P.chunks;
+    c.hk = it % P.H_kv;
+    c.s = it / P.H_kv;
+    int pl = P.prefix_len[c.s];
+    if (pl < 0 || pl > P.pl_max) {
+        flags |= HAWK_DEV_BAD_PREFIX;
+        pl = max(0, min(pl, P.pl_max));
+    }
+    c.pl = pl;
+    c.ntiles = (pl + P.K + TK - 1) / TK;
+    c.row_base = (c.s * P.H_kv + c.hk) * P.L_cap;
+}
+
+// Moves the cursor to the next tile at or after its position that holds visible keys; false when
+// the share is exhausted.  Tiles past a stream's last visible key are skipped without a load.
+template <int TK>
+__device__ __forceinline__ bool seek_valid(Cursor &c, long long f_end, const AttnParams &P, int &flags)
+{
+    while (c.f < f_end) {
+        if (c.tile < c.ntiles) return true;
+        c.f += P.tiles_per_item - c.tile;  // first tile of the next item
+        if (c.f >= f_end) return false;
+        decode_item<TK>(c, P, flags);
+    }
+    return false;
+}
+
+template <int TK>
+__device__ __forceinline__ void step(Cursor &c, long long f_end, const AttnParams &P, int &flags)
+{
+    ++c.f;
+    ++c.tile;
+    if (c.tile == P.tiles_per_item && c.f < f_end) decode_item<TK>(c, P, flags);
+}
+
+__device__ __forceinline__ uint32_t movmatrix_trans(uint32_t x)
+{
+    uint32_t y;
+    asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(y) : "r"(x));
+    return y;
+}
+
+// NQT = number of 8-query column tiles: 1 when an item has at most 8 query rows, else 2.
+template <int D, int NQT>
+__global__ void __launch_bounds__(kThreads, 1) attn_kernel(const __grid_constant__ CUtensorMap map_k,
+                                                           const __grid_constant__ CUtensorMap map_v,
+                                                           const AttnParams P)
 {
     using C = AttnCfg<D>;
+    constexpr int TK = C::kTileKeys;
+    constexpr int KB = TK / 16;  // 16-key MMA blocks per tile
+    constexpr int DB = D / 16;   // 16-wide blocks of the head dimension
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-    uint8_t *stage_base = smem;
-    float *merge = reinterpret_cast<float *>(smem);  // reused once every tile has been consumed
-    uint64_t *full_bar = reinterpret_cast<uint64_t *>(smem + C::kStages * C::kStageBytes);
-    uint64_t *empty_bar = full_bar + C::kStages;
-    volatile int *abort_flag = reinterpret_cast<volatile int *>(empty_bar + C::kStages);
+    uint64_t *bars = reinterpret_cast<uint64_t *>(smem + kWarps * kStages * kStageBytes);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-
-    // ---- which item
-    int item = blockIdx.x;
-    const int sp = item % P.nsplit;
-    item /= P.nsplit;
-    const int chunk = item % P.chunks;
-    item /= P.chunks;
-    const int hk = item % P.H_kv;
-    const int s = item / P.H_kv;
-    const int group = P.H / P.H_kv;
-    const int h0 = hk * group + chunk * P.chunk_heads;                       // first query head of the item
-    const int nheads = min(P.chunk_heads, group - chunk * P.chunk_heads);    // heads in this chunk
-    const int nrows = nheads * P.K;
-
-    int pl = P.prefix_len[s];
-    if (pl < 0 || pl > P.L_cap - P.K) {
-        if (tid == 0 && P.dev_status) atomicOr(P.dev_status, HAWK_DEV_BAD_PREFIX);
-        pl = max(0, min(pl, P.L_cap - P.K));
-    }
-    const int n_total = pl + P.K;  // keys any query of this stream can see
-    const int tiles = (n_total + kTileKeys - 1) / kTileKeys;
-    const int tiles_per_split = (tiles + P.nsplit - 1) / P.nsplit;
-    const int t_begin = sp * tiles_per_split;
-    const int t_end = min(tiles, t_begin + tiles_per_split);
-    const int row_base = (s * P.H_kv + hk) * P.L_cap;  // first cache row of this (stream, kv head)
-
+    // No allow_dependent_launch() here: with the merge kernel's blocks resident and waiting from the
+    // start, this kernel measured 10 % slower; the merge kernel is released when the blocks exit.
     if (tid == 0) {
-        for (int i = 0; i < C::kStages; ++i) {
-            mbar_init(&full_bar[i], 1);
-            mbar_init(&empty_bar[i], kConsumerWarps);
-        }
-        *abort_flag = 0;
+        for (int i = 0; i < kWarps * kStages; ++i) mbar_init(&bars[i], 1);
         fence_mbar_init();
+        fence_proxy_async();
     }
-    __syncthreads();
+    __syncthreads();  // the only block-wide synchronisation: from here on every warp runs alone
+    grid_dependency_wait();
 
-    if (warp == kConsumerWarps) {
-        // =========================== producer warp: one lane issues every tile load
+    const int w = blockIdx.x * kWarps + warp;
+    if (w >= P.workers) return;
+    uint8_t *ring = smem + warp * kStages * kStageBytes;
+    uint64_t *full_bar = bars + warp * kStages;
+    const uint32_t ring_u32 = smem_u32(ring);
+
+    const long long T = P.total_tiles;
+    const long long f_begin = share_begin(w, T, P.workers), f_end = share_begin(w + 1, T, P.workers);
+    int flags = 0;
+
+    uint64_t policy = 0;
+    if (lane == 0) {
+        prefetch_tensormap(&map_k);
+        prefetch_tensormap(&map_v);
+        policy = l2_policy_evict_first();
+    }
+
+    // ---- issue side: runs up to kStages tiles ahead of the consume side
+    Cursor ci;
+    ci.f = f_begin;
+    decode_item<TK>(ci, P, flags);
+    auto issue = [&](const Cursor &c, int st) {
         if (lane == 0) {
-            prefetch_tensormap(&map_k);
-            prefetch_tensormap(&map_v);
-            const uint64_t policy = l2_policy_evict_first();
-            int st = 0;
-            uint32_t ph = 0;
-            bool ok = true;
-            int issued = 0;
-            uint32_t armed_parity[C::kStages];
-            for (int t = t_begin; t < t_end && ok; ++t) {
-                if (issued >= C::kStages) ok = mbar_wait(&empty_bar[st], ph ^ 1u, abort_flag);
-                if (!ok) break;
-                uint8_t *kd = stage_base + st * C::kStageBytes;
-                uint8_t *vd = kd + C::kHalves * C::kSubTileBytes;
-                mbar_arrive_expect_tx(&full_bar[st], C::kStageBytes);
-                armed_parity[st] = ph;
-                const int y = row_base + t * kTileKeys;
+            uint8_t *kd = ring + st * kStageBytes;
+            uint8_t *vd = kd + C::kHalves * C::kSubTileBytes;
+            mbar_arrive_expect_tx(&full_bar[st], kStageBytes);
+            const int y = c.row_base + c.tile * TK;
 #pragma unroll
-                for (int hf = 0; hf < C::kHalves; ++hf) {
-                    tma_load_2d_hint(kd + hf * C::kSubTileBytes, &map_k, hf * 64, y, &full_bar[st], policy);
-                    tma_load_2d_hint(vd + hf * C::kSubTileBytes, &map_v, hf * 64, y, &full_bar[st], policy);
-                }
-                ++issued;
-                if (++st == C::kStages) {
-                    st = 0;
-                    ph ^= 1u;
-                }
-            }
-            if (!ok) {
-                *abort_flag = 1;
-                if (P.dev_status) atomicOr(P.dev_status, HAWK_DEV_TIMEOUT);
-                // let the copies already issued land (bounded) before the block can retire
-                for (int i = 0; i < C::kStages && i < issued; ++i) mbar_wait(&full_bar[i], armed_parity[i], nullptr);
+            for (int hf = 0; hf < C::kHalves; ++hf) {
+                tma_load_2d_hint(kd + hf * C::kSubTileBytes, &map_k, hf * 64, y, &full_bar[st], policy);
+                tma_load_2d_hint(vd + hf * C::kSubTileBytes, &map_v, hf * 64, y, &full_bar[st], policy);
             }
         }
-        return;  // consumers only use named barrier 1 from here on
-    }
-
-    // =========================== consumer warps
-    const int g = lane >> 2, tq = lane & 3;  // fragment row / column-pair index
-    // row r of the 16-row query operand: head h0 + r / K, draft position r % K (rows >= nrows are padding)
-    const int r0 = g, r1 = g + 8;
-    const int i0 = r0 % P.K, i1 = r1 % P.K;
-    const bool v0 = r0 < nrows, v1 = r1 < nrows;
-    const int lim0 = pl + i0 + 1, lim1 = pl + i1 + 1;  // visible keys: j < lim
-
-    // Q fragments (A operand, 16 x D), straight from global memory
-    uint32_t qa[D / 16][4];
-    {
-        const __nv_bfloat16 *q0 = P.q + ((static_cast<size_t>(s) * P.K + i0) * P.H + (h0 + r0 / P.K)) * D;
-        const __nv_bfloat16 *q1 = P.q + ((static_cast<size_t>(s) * P.K + i1) * P.H + (h0 + r1 / P.K)) * D;
+    };
+    int in_flight = 0;  // stages armed and not yet consumed
 #pragma unroll
-        for (int kk = 0; kk < D / 16; ++kk) {
-            const int d = kk * 16 + 2 * tq;
-            qa[kk][0] = v0 ? *reinterpret_cast<const uint32_t *>(q0 + d) : 0u;
-            qa[kk][1] = v1 ? *reinterpret_cast<const uint32_t *>(q1 + d) : 0u;
-            qa[kk][2] = v0 ? *reinterpret_cast<const uint32_t *>(q0 + d + 8) : 0u;
-            qa[kk][3] = v1 ? *reinterpret_cast<const uint32_t *>(q1 + d + 8) : 0u;
+    for (int i = 0; i < kStages; ++i) {
+        if (seek_valid<TK>(ci, f_end, P, flags)) {
+            issue(ci, i);
+            step<TK>(ci, f_end, P, flags);
+            ++in_flight;
         }
     }
 
-    float o[D / 8][4];
-#pragma unroll
-    for (int c = 0; c < D / 8; ++c) o[c][0] = o[c][1] = o[c][2] = o[c][3] = 0.f;
-    float m0 = -CUDART_INF_F, m1 = -CUDART_INF_F, l0 = 0.f, l1 = 0.f;  // running max (log2 units) and sum
+    // ---- consume side.  Fragment coordinates of this thread: g = lane / 4, tq = lane % 4.
+    //   S^T block (16 keys x 8 queries): keys g and g + 8, queries 2tq and 2tq + 1 of the column tile
+    //   O^T block (16 dims x 8 queries): dims g and g + 8,  queries 2tq and 2tq + 1
+    const int g = lane >> 2, tq = lane & 3;
+    const int lm_mi = lane >> 3, lm_r = lane & 7;  // ldmatrix: this lane addresses row lm_r of matrix lm_mi
+    const int group = P.H / P.H_kv;
 
+    // byte offsets inside a stage of the ldmatrix rows this lane addresses (128-byte swizzle: the
+    // 16-byte chunk index is XOR-ed with the row index modulo 8)
+    //   K (plain):      matrices (keys 0-7, chunk 2kk), (keys 8-15, 2kk), (keys 0-7, 2kk+1), (keys 8-15, 2kk+1)
+    //   V (transposed): matrices (keys 0-7, chunk 2db), (keys 0-7, 2db+1), (keys 8-15, 2db), (keys 8-15, 2db+1)
+    uint32_t k_off[DB], v_off[DB];
+#pragma unroll
+    for (int kk = 0; kk < DB; ++kk) {
+        const int kc = 2 * kk + (lm_mi >> 1), vc = 2 * kk + (lm_mi & 1);
+        k_off[kk] = (kc >> 3) * C::kSubTileBytes + ((lm_mi & 1) * 8 + lm_r) * 128 + (((kc & 7) ^ lm_r) << 4);
+        v_off[kk] = (vc >> 3) * C::kSubTileBytes + ((lm_mi >> 1) * 8 + lm_r) * 128 + (((vc & 7) ^ lm_r) << 4);
+    }
+
+    uint32_t qb[NQT][DB][2];  // Q^T as the 16 x 8 operand: query row = column tile * 8 + g
+    float ot[NQT][DB][4];     // O^T accumulators
+    float mrun[NQT][2], lrun[NQT][2];  // running max (log2 units) and this thread's share of the running sum
+    int lim[NQT][2];          // visible keys of the queries in this thread's columns: j < lim
+    int cur_item = -1, h0 = 0, nrows = 0, seg_pl = 0, seg_s = 0;
+    long long seg_start = 0;
+
+    // Writes the finished segment: final bf16 rows if the share held the whole item, else an fp32 partial.
+    auto flush = [&]() {
+        if (cur_item < 0) return;
+#pragma unroll
+        for (int nq = 0; nq < NQT; ++nq)
+#pragma unroll
+            for (int c = 0; c < 2; ++c) {
+                float l = lrun[nq][c];
+                l += __shfl_xor_sync(0xffffffffu, l, 4);
+                l += __shfl_xor_sync(0xffffffffu, l, 8);
+                l += __shfl_xor_sync(0xffffffffu, l, 16);
+                lrun[nq][c] = l;
+            }
+        const long long a = static_cast<long long>(cur_item) * P.tiles_per_item, b = a + P.tiles_per_item;
+        const bool complete = a >= f_begin && b <= f_end;
+        if (complete) {
+#pragma unroll
+            for (int nq = 0; nq < NQT; ++nq) {
+                const float inv0 = 1.f / lrun[nq][0], inv1 = 1.f / lrun[nq][1];
+                const int r = nq * 8 + g;  // after the transposes below this thread holds query row r
+                const bool valid = r < nrows;
+                __nv_bfloat16 *dst =
+                    P.out + ((static_cast<size_t>(seg_s) * P.K + r % P.K) * P.H + (h0 + r / P.K)) * D + 2 * tq;
+#pragma unroll
+                for (int db = 0; db < DB; ++db) {
+                    // (dims g / g+8) x (queries 2tq, 2tq+1)  ->  (query g) x (dims 2tq, 2tq+1 / +8)
+                    const uint32_t lo = movmatrix_trans(pack_bf16(ot[nq][db][0] * inv0, ot[nq][db][1] * inv1));
+                    const uint32_t hi = movmatrix_trans(pack_bf16(ot[nq][db][2] * inv0, ot[nq][db][3] * inv1));
+                    if (valid) {
+                        *reinterpret_cast<uint32_t *>(dst + db * 16) = lo;
+                        *reinterpret_cast<uint32_t *>(dst + db * 16 + 8) = hi;
+                    }
+                }
+            }
+        } else {
+            const int slot = seg_start == f_begin ? 0 : 1;
+            float *ps = P.part + (static_cast<size_t>(w) * 2 + slot) * 16 * (D + 2);
+#pragma unroll
+            for (int nq = 0; nq < NQT; ++nq)
+#pragma unroll
+                for (int c = 0; c < 2; ++c) {
+                    const int r = nq * 8 + 2 * tq + c;
+                    if (r < nrows) {
+                        float *pr = ps + r * D;
+#pragma unroll
+                        for (int db = 0; db < DB; ++db) {
+                            pr[db * 16 + g] = ot[nq][db][c];
+                            pr[db * 16 + 8 + g] = ot[nq][db][2 + c];
+                        }
+                        if (g == 0)
+                            *reinterpret_cast<float2 *>(ps + 16 * D + 2 * r) = make_float2(mrun[nq][c], lrun[nq][c]);
+                    }
+                }
+        }
+    };
+
+    // Q^T operand of one item, straight from global memory (rows past the item's last are zero)
+    uint32_t qn[NQT][DB][2];  // the same for the item that follows in the share, fetched ahead
+    int qn_item = -1;
+    auto load_q = [&](uint32_t (&dst)[NQT][DB][2], int item) {
+        int it = item;
+        const int chunk = it % P.chunks;
+        it /= P.chunks;
+        const int hk = it % P.H_kv, s = it / P.H_kv;
+        const int hq0 = hk * group + chunk * P.chunk_heads;
+        const int rows = min(P.chunk_heads, group - chunk * P.chunk_heads) * P.K;
+#pragma unroll
+        for (int nq = 0; nq < NQT; ++nq) {
+            const int r = nq * 8 + g;  // query row whose values this thread feeds into the operand
+            const bool valid = r < rows;
+            const __nv_bfloat16 *qr =
+                P.q + ((static_cast<size_t>(s) * P.K + r % P.K) * P.H + (hq0 + r / P.K)) * D + 2 * tq;
+#pragma unroll
+            for (int kk = 0; kk < DB; ++kk) {
+                dst[nq][kk][0] = valid ? *reinterpret_cast<const uint32_t *>(qr + kk * 16) : 0u;
+                dst[nq][kk][1] = valid ? *reinterpret_cast<const uint32_t *>(qr + kk * 16 + 8) : 0u;
+            }
+        }
+    };
+
+    Cursor cc;
+    cc.f = f_begin;
+    decode_item<TK>(cc, P, flags);
     int st = 0;
     uint32_t ph = 0;
     bool ok = true;
-    const uint32_t stage_u32 = smem_u32(stage_base);
-    // ldmatrix row addressing: lane -> (matrix mi = lane / 8, row lane % 8)
-    const int lm_mi = lane >> 3, lm_r = lane & 7;
-
-    for (int t = t_begin; t < t_end; ++t) {
-        ok = mbar_wait(&full_bar[st], ph, abort_flag);
-        if (!ok) break;
-        const uint32_t kbase = stage_u32 + st * C::kStageBytes;
-        const uint32_t vbase = kbase + C::kHalves * C::kSubTileBytes;
-        const int key0 = t * kTileKeys + warp * kKeysPerWarp;  // first key of this warp's slice
-
-        if (key0 < n_total) {
-            // ---- scores S = Q K^T for 16 keys: two 8-key column tiles
-            float sc[2][4];
+    while (seek_valid<TK>(cc, f_end, P, flags)) {
+        if (cc.item != cur_item) {
+            // ---- a new segment: write the previous one, fetch this item's queries, reset the state
+            flush();
+            cur_item = cc.item;
+            seg_start = cc.f;
+            seg_pl = cc.pl;
+            seg_s = cc.s;
+            h0 = cc.hk * group + cc.chunk * P.chunk_heads;
+            const int nheads = min(P.chunk_heads, group - cc.chunk * P.chunk_heads);
+            nrows = nheads * P.K;
+            if (qn_item == cc.item) {
 #pragma unroll
-            for (int nt = 0; nt < 2; ++nt) sc[nt][0] = sc[nt][1] = sc[nt][2] = sc[nt][3] = 0.f;
+                for (int nq = 0; nq < NQT; ++nq)
 #pragma unroll
-            for (int kk = 0; kk < D / 16; ++kk) {
-                // matrices: (keys 0-7, d lo), (keys 0-7, d hi), (keys 8-15, d lo), (keys 8-15, d hi)
-                const int krow = warp * kKeysPerWarp + (lm_mi >> 1) * 8 + lm_r;
-                const int chunk16 = kk * 2 + (lm_mi & 1);  // 16-byte column chunk 0 .. D/8-1
-                const uint32_t addr = kbase + (chunk16 >> 3) * C::kSubTileBytes + krow * 128 +
-                                      (((chunk16 & 7) ^ (krow & 7)) << 4);
-                uint32_t kb[4];
-                ldmatrix_x4(kb, addr);
-                mma_bf16_16816(sc[0], qa[kk], kb[0], kb[1]);
-                mma_bf16_16816(sc[1], qa[kk], kb[2], kb[3]);
+                    for (int kk = 0; kk < DB; ++kk) {
+                        qb[nq][kk][0] = qn[nq][kk][0];
+                        qb[nq][kk][1] = qn[nq][kk][1];
+                    }
+            } else {
+                load_q(qb, cc.item);
             }
-            // ---- causal mask inside the block (only tiles that reach past the prefix)
-            if (key0 + kKeysPerWarp > pl) {
+            // the next item of the share follows in a few tiles: fetch its queries now, off the critical path
+            qn_item = cc.item + 1;
+            if (static_cast<long long>(qn_item) * P.tiles_per_item < f_end) load_q(qn, qn_item);
+            else qn_item = -1;
 #pragma unroll
-                for (int nt = 0; nt < 2; ++nt) {
-                    const int j = key0 + nt * 8 + 2 * tq;
-                    if (j >= lim0) sc[nt][0] = -CUDART_INF_F;
-                    if (j + 1 >= lim0) sc[nt][1] = -CUDART_INF_F;
-                    if (j >= lim1) sc[nt][2] = -CUDART_INF_F;
-                    if (j + 1 >= lim1) sc[nt][3] = -CUDART_INF_F;
+            for (int nq = 0; nq < NQT; ++nq) {
+#pragma unroll
+                for (int db = 0; db < DB; ++db) ot[nq][db][0] = ot[nq][db][1] = ot[nq][db][2] = ot[nq][db][3] = 0.f;
+#pragma unroll
+                for (int c = 0; c < 2; ++c) {
+                    mrun[nq][c] = -CUDART_INF_F;
+                    lrun[nq][c] = 0.f;
+                    lim[nq][c] = cc.pl + (nq * 8 + 2 * tq + c) % P.K + 1;
                 }
             }
-            // ---- running softmax (log2 domain), quad shuffles for the row maximum
-            float mx0 = fmaxf(fmaxf(sc[0][0], sc[0][1]), fmaxf(sc[1][0], sc[1][1]));
-            float mx1 = fmaxf(fmaxf(sc[0][2], sc[0][3]), fmaxf(sc[1][2], sc[1][3]));
-            mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 1));
-            mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 2));
-            mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 1));
-            mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 2));
-            const float mn0 = fmaxf(m0, mx0 * P.scale_log2), mn1 = fmaxf(m1, mx1 * P.scale_log2);
+        }
+        const int pl = seg_pl;
+        const int n_total = pl + P.K;  // keys any query of this stream can see
+        const int tile_key0 = cc.tile * TK;
+
+        ok = mbar_wait(&full_bar[st], ph, nullptr);
+        if (!ok) break;
+        const uint32_t kbase = ring_u32 + st * kStageBytes;
+        const uint32_t vbase = kbase + C::kHalves * C::kSubTileBytes;
+
+        // ---- scores S^T = K Q^T for the whole tile
+        float sc[NQT][KB][4];
+#pragma unroll
+        for (int kb = 0; kb < KB; ++kb) {
+#pragma unroll
+            for (int nq = 0; nq < NQT; ++nq) sc[nq][kb][0] = sc[nq][kb][1] = sc[nq][kb][2] = sc[nq][kb][3] = 0.f;
+#pragma unroll
+            for (int kk = 0; kk < DB; ++kk) {
+                uint32_t ka[4];
+                ldmatrix_x4(ka, kbase + kb * 2048 + k_off[kk]);
+#pragma unroll
+                for (int nq = 0; nq < NQT; ++nq) mma_bf16_16816(sc[nq][kb], ka, qb[nq][kk][0], qb[nq][kk][1]);
+            }
+        }
+        // ---- causal mask inside the block, which also hides the cache rows past the last visible key
+        if (tile_key0 + TK > pl) {
+#pragma unroll
+            for (int kb = 0; kb < KB; ++kb) {
+                const int j0 = tile_key0 + kb * 16 + g, j1 = j0 + 8;
+#pragma unroll
+                for (int nq = 0; nq < NQT; ++nq) {
+                    if (j0 >= lim[nq][0]) sc[nq][kb][0] = -CUDART_INF_F;
+                    if (j0 >= lim[nq][1]) sc[nq][kb][1] = -CUDART_INF_F;
+                    if (j1 >= lim[nq][0]) sc[nq][kb][2] = -CUDART_INF_F;
+                    if (j1 >= lim[nq][1]) sc[nq][kb][3] = -CUDART_INF_F;
+                }
+            }
+        }
+        // ---- running softmax per query column (log2 domain): one max reduction and one rescale per tile
+        uint32_t pb[NQT][KB][2];  // P^T as the 16 x 8 operand of the second product
+#pragma unroll
+        for (int nq = 0; nq < NQT; ++nq) {
+            float mx0 = -CUDART_INF_F, mx1 = -CUDART_INF_F;
+#pragma unroll
+            for (int kb = 0; kb < KB; ++kb) {
+                mx0 = fmaxf(mx0, fmaxf(sc[nq][kb][0], sc[nq][kb][2]));
+                mx1 = fmaxf(mx1, fmaxf(sc[nq][kb][1], sc[nq][kb][3]));
+            }
+#pragma unroll
+            for (int o = 4; o < 32; o <<= 1) {
+                mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, o));
+                mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, o));
+            }
+            const float mn0 = fmaxf(mrun[nq][0], mx0 * P.scale_log2), mn1 = fmaxf(mrun[nq][1], mx1 * P.scale_log2);
             const float mu0 = mn0 == -CUDART_INF_F ? 0.f : mn0, mu1 = mn1 == -CUDART_INF_F ? 0.f : mn1;
-            const float a0 = fast_exp2(m0 - mu0), a1 = fast_exp2(m1 - mu1);
-            m0 = mn0;
-            m1 = mn1;
-            float p[2][4];
+            const float a0 = fast_exp2(mrun[nq][0] - mu0), a1 = fast_exp2(mrun[nq][1] - mu1);
+            mrun[nq][0] = mn0;
+            mrun[nq][1] = mn1;
+            float s0 = 0.f, s1 = 0.f;
 #pragma unroll
-            for (int nt = 0; nt < 2; ++nt) {
-                p[nt][0] = fast_exp2(fmaf(sc[nt][0], P.scale_log2, -mu0));
-                p[nt][1] = fast_exp2(fmaf(sc[nt][1], P.scale_log2, -mu0));
-                p[nt][2] = fast_exp2(fmaf(sc[nt][2], P.scale_log2, -mu1));
-                p[nt][3] = fast_exp2(fmaf(sc[nt][3], P.scale_log2, -mu1));
+            for (int kb = 0; kb < KB; ++kb) {
+                const float p0 = fast_exp2(fmaf(sc[nq][kb][0], P.scale_log2, -mu0));
+                const float p1 = fast_exp2(fmaf(sc[nq][kb][1], P.scale_log2, -mu1));
+                const float p2 = fast_exp2(fmaf(sc[nq][kb][2], P.scale_log2, -mu0));
+                const float p3 = fast_exp2(fmaf(sc[nq][kb][3], P.scale_log2, -mu1));
+                s0 += p0 + p2;
+                s1 += p1 + p3;
+                // (key g / g+8) x (queries 2tq, 2tq+1)  ->  (keys 2tq, 2tq+1 / +8) x (query g)
+                pb[nq][kb][0] = movmatrix_trans(pack_bf16(p0, p1));
+                pb[nq][kb][1] = movmatrix_trans(pack_bf16(p2, p3));
             }
-            l0 = l0 * a0 + ((p[0][0] + p[0][1]) + (p[1][0] + p[1][1]));
-            l1 = l1 * a1 + ((p[0][2] + p[0][3]) + (p[1][2] + p[1][3]));
+            lrun[nq][0] = lrun[nq][0] * a0 + s0;
+            lrun[nq][1] = lrun[nq][1] * a1 + s1;
 #pragma unroll
-            for (int c = 0; c < D / 8; ++c) {
-                o[c][0] *= a0;
-                o[c][1] *= a0;
-                o[c][2] *= a1;
-                o[c][3] *= a1;
+            for (int db = 0; db < DB; ++db) {
+                ot[nq][db][0] *= a0;
+                ot[nq][db][1] *= a1;
+                ot[nq][db][2] *= a0;
+                ot[nq][db][3] *= a1;
             }
-            // P as the A operand of P.V (16 rows x 16 keys)
-            uint32_t pa[4];
-            pa[0] = pack_bf16(p[0][0], p[0][1]);
-            pa[1] = pack_bf16(p[0][2], p[0][3]);
-            pa[2] = pack_bf16(p[1][0], p[1][1]);
-            pa[3] = pack_bf16(p[1][2], p[1][3]);
-            // keys at or past n_total hold whatever the cache holds: zero them so 0 * NaN cannot appear
-            const bool ragged = key0 + kKeysPerWarp > n_total;
-            const int kleft = n_total - key0;  // valid keys in this slice when ragged
+        }
+        // ---- O^T += V^T P^T.  Cache rows at or past n_total hold whatever the cache holds: zero
+        // them so that 0 * NaN cannot appear.
+        const bool ragged = tile_key0 + TK > n_total;
 #pragma unroll
-            for (int c = 0; c < D / 8; c += 2) {
-                // matrices: (keys 0-7, chunk c), (keys 8-15, chunk c), (keys 0-7, chunk c+1), (keys 8-15, chunk c+1)
-                const int krow = warp * kKeysPerWarp + (lm_mi & 1) * 8 + lm_r;
-                const int chunk16 = c + (lm_mi >> 1);
-                const uint32_t addr = vbase + (chunk16 >> 3) * C::kSubTileBytes + krow * 128 +
-                                      (((chunk16 & 7) ^ (krow & 7)) << 4);
-                uint32_t vb[4];
-                ldmatrix_x4_trans(vb, addr);
-                if (ragged) {
-                    // register 0/2: keys 2tq, 2tq+1; register 1/3: keys 2tq+8, 2tq+9 (low half = first key)
+        for (int kb = 0; kb < KB; ++kb) {
+            const int kleft = n_total - (tile_key0 + kb * 16);  // visible keys in this 16-key block
+            if (ragged && kleft <= 0) break;
+#pragma unroll
+            for (int db = 0; db < DB; ++db) {
+                uint32_t va[4];
+                ldmatrix_x4_trans(va, vbase + kb * 2048 + v_off[db]);
+                if (ragged && kleft < 16) {
+                    // registers 0/1: keys 2tq, 2tq+1; registers 2/3: keys 2tq+8, 2tq+9 (low half = first key)
                     const int ka = 2 * tq, kb2 = 2 * tq + 8;
                     const uint32_t ma = (ka < kleft ? 0x0000ffffu : 0u) | (ka + 1 < kleft ? 0xffff0000u : 0u);
                     const uint32_t mb = (kb2 < kleft ? 0x0000ffffu : 0u) | (kb2 + 1 < kleft ? 0xffff0000u : 0u);
-                    vb[0] &= ma;
-                    vb[2] &= ma;
-                    vb[1] &= mb;
-                    vb[3] &= mb;
+                    va[0] &= ma;
+                    va[1] &= ma;
+                    va[2] &= mb;
+                    va[3] &= mb;
                 }
-                mma_bf16_16816(o[c], pa, vb[0], vb[1]);
-                mma_bf16_16816(o[c + 1], pa, vb[2], vb[3]);
+#pragma unroll
+                for (int nq = 0; nq < NQT; ++nq) mma_bf16_16816(ot[nq][db], va, pb[nq][kb][0], pb[nq][kb][1]);
             }
         }
         __syncwarp();
-        if (lane == 0) mbar_arrive(&empty_bar[st]);
-        if (++st == C::kStages) {
+        --in_flight;
+        // ---- the stage is free again: load the next tile of the share into it
+        if (seek_valid<TK>(ci, f_end, P, flags)) {
+            fence_proxy_async();  // the warp's reads of the stage come before the copy that overwrites it
+            issue(ci, st);
+            step<TK>(ci, f_end, P, flags);
+            ++in_flight;
+        }
+        step<TK>(cc, f_end, P, flags);
+        if (++st == kStages) {
             st = 0;
             ph ^= 1u;
         }
     }
-    if (!ok) {
-        if (lane == 0) {
-            *abort_flag = 1;
-            if (P.dev_status) atomicOr(P.dev_status, HAWK_DEV_TIMEOUT);
+    if (ok) {
+        flush();
+    } else {
+        flags |= HAWK_DEV_TIMEOUT;
+        // let the copies still in flight land (bounded) before the block can retire
+        for (int i = 0; i < in_flight; ++i) {
+            mbar_wait(&full_bar[st], ph, nullptr);
+            if (++st == kStages) {
+                st = 0;
+                ph ^= 1u;
+            }
         }
     }
-
-    // ---- merge the four warps' partial softmax states through shared memory
-    l0 += __shfl_xor_sync(0xffffffffu, l0, 1);
-    l0 += __shfl_xor_sync(0xffffffffu, l0, 2);
-    l1 += __shfl_xor_sync(0xffffffffu, l1, 1);
-    l1 += __shfl_xor_sync(0xffffffffu, l1, 2);
-    asm volatile("bar.sync 1, %0;" ::"n"(kConsumerWarps * 32) : "memory");  // all slices read: ring is free
-    float *mw = merge + warp * 16 * (D + 2);
-#pragma unroll
-    for (int c = 0; c < D / 8; ++c) {
-        const int d = c * 8 + 2 * tq;
-        *reinterpret_cast<float2 *>(mw + r0 * (D + 2) + d) = make_float2(o[c][0], o[c][1]);
-        *reinterpret_cast<float2 *>(mw + r1 * (D + 2) + d) = make_float2(o[c][2], o[c][3]);
-    }
-    if (tq == 0) {
-        mw[r0 * (D + 2) + D] = m0;
-        mw[r0 * (D + 2) + D + 1] = l0;
-        mw[r1 * (D + 2) + D] = m1;
-        mw[r1 * (D + 2) + D + 1] = l1;
-    }
-    asm volatile("bar.sync 1, %0;" ::"n"(kConsumerWarps * 32) : "memory");
-
-    // every consumer thread finishes a strided set of (row, column pair) outputs
-    constexpr int kPairs = D / 2;
-    for (int idx = tid; idx < nrows * kPairs; idx += kConsumerWarps * 32) {
-        const int r = idx / kPairs, d = (idx - r * kPairs) * 2;
-        float mm = -CUDART_INF_F;
-#pragma unroll
-        for (int w = 0; w < kConsumerWarps; ++w) mm = fmaxf(mm, merge[(w * 16 + r) * (D + 2) + D]);
-        const float mu = mm == -CUDART_INF_F ? 0.f : mm;
-        float ll = 0.f, ox = 0.f, oy = 0.f;
-#pragma unroll
-        for (int w = 0; w < kConsumerWarps; ++w) {
-            const float *rw = merge + (w * 16 + r) * (D + 2);
-            const float f = fast_exp2(rw[D] - mu);
-            ll += rw[D + 1] * f;
-            const float2 ov = *reinterpret_cast<const float2 *>(rw + d);
-            ox += ov.x * f;
-            oy += ov.y * f;
-        }
-        const int h = h0 + r / P.K, i = r % P.K;
-        if (P.nsplit == 1) {
-            const float inv = 1.f / ll;
-            __nv_bfloat162 ob = __floats2bfloat162_rn(ox * inv, oy * inv);
-            *reinterpret_cast<__nv_bfloat162 *>(P.out + ((static_cast<size_t>(s) * P.K + i) * P.H + h) * D + d) = ob;
-        } else {
-            const size_t prow = ((static_cast<size_t>(s) * P.H + h) * P.K + i) * P.nsplit + sp;
-            *reinterpret_cast<float2 *>(P.part_o + prow * D + d) = make_float2(ox, oy);
-            if (d == 0) *reinterpret_cast<float2 *>(P.part_ml + prow * 2) = make_float2(mm, ll);
-        }
-    }
+    if (flags && lane == 0 && P.dev_status) atomicOr(P.dev_status, flags);
 }
 
-// Merges the per-split partial results: one warp per (stream, head, draft position) row.
+// Merges the partial results of every item whose tiles were spread over several shares:
+// one warp per (item, query row of the item), lanes across the head dimension.
 template <int D>
-__global__ void attn_combine_kernel(const float *part_o, const float *part_ml, __nv_bfloat16 *out, int rows_total,
-                                    int K, int H, int nsplit)
+__global__ void attn_combine_kernel(const AttnParams P, int items, int rows_per_item)
 {
-    const int row = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;  // (s*H + h)*K + i
+    constexpr int TK = AttnCfg<D>::kTileKeys;
+    allow_dependent_launch();
+    grid_dependency_wait();  // every thread waits, so this grid cannot retire before the attention kernel has
+    const int wid = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const int lane = threadIdx.x & 31;
-    if (row >= rows_total) return;
-    float mm = -CUDART_INF_F;
-    for (int sp = 0; sp < nsplit; ++sp) mm = fmaxf(mm, part_ml[(static_cast<size_t>(row) * nsplit + sp) * 2]);
-    const float mu = mm == -CUDART_INF_F ? 0.f : mm;
+    const int item = wid / rows_per_item, r = wid - item * rows_per_item;
+    if (item >= items) return;
+    const long long T = P.total_tiles;
+    const long long a = static_cast<long long>(item) * P.tiles_per_item, b = a + P.tiles_per_item;
+    const int g_first = owner(a, T, P.workers), g_last = owner(b - 1, T, P.workers);
+    if (g_first == g_last) return;  // one share held the whole item and wrote the result itself
+    int it = item;
+    const int chunk = it % P.chunks;
+    it /= P.chunks;
+    const int hk = it % P.H_kv, s = it / P.H_kv;
+    const int group = P.H / P.H_kv;
+    const int nheads = min(P.chunk_heads, group - chunk * P.chunk_heads);
+    if (r >= nheads * P.K) return;
+    const int pl = max(0, min(P.prefix_len[s], P.pl_max));
+    const int ntiles = (pl + P.K + TK - 1) / TK;
+
     constexpr int PER = D / 32;
     float acc[PER];
 #pragma unroll
     for (int c = 0; c < PER; ++c) acc[c] = 0.f;
-    float ll = 0.f;
-    for (int sp = 0; sp < nsplit; ++sp) {
-        const size_t pr = static_cast<size_t>(row) * nsplit + sp;
-        const float f = fast_exp2(part_ml[pr * 2] - mu);
-        ll += part_ml[pr * 2 + 1] * f;
-        if (PER == 2) {
-            const float2 v = *reinterpret_cast<const float2 *>(part_o + pr * D + lane * 2);
-            acc[0] += v.x * f;
-            acc[1] += v.y * f;
+    float mm = -CUDART_INF_F, ll = 0.f;
+    for (int gg = g_first; gg <= g_last; ++gg) {
+        const long long sb = share_begin(gg, T, P.workers);
+        const long long seg_begin = sb > a ? sb : a;
+        if (seg_begin - a >= ntiles) break;  // this share and all later ones saw no visible key of the item
+        const int slot = a <= sb ? 0 : 1;
+        const float *slot_base = P.part + (static_cast<size_t>(gg) * 2 + slot) * 16 * (D + 2);
+        const float *ps = slot_base + r * D + lane * PER;  // 16-byte aligned for D = 128, 8-byte for D = 64
+        const float2 ml = *reinterpret_cast<const float2 *>(slot_base + 16 * D + 2 * r);
+        float v[PER];
+        if constexpr (PER == 2) {
+            const float2 t = *reinterpret_cast<const float2 *>(ps);
+            v[0] = t.x;
+            v[1] = t.y;
         } else {
-            const float4 v = *reinterpret_cast<const float4 *>(part_o + pr * D + lane * 4);
-            acc[0] += v.x * f;
-            acc[1] += v.y * f;
-            acc[2] += v.z * f;
-            acc[3] += v.w * f;
+            const float4 t = *reinterpret_cast<const float4 *>(ps);
+            v[0] = t.x;
+            v[1] = t.y;
+            v[PER - 2] = t.z;
+            v[PER - 1] = t.w;
         }
+        const float mn = fmaxf(mm, ml.x);
+        const float mu = mn == -CUDART_INF_F ? 0.f : mn;
+        const float f_old = fast_exp2(mm - mu), f_new = fast_exp2(ml.x - mu);
+        mm = mn;
+        ll = ll * f_old + ml.y * f_new;
+#pragma unroll
+        for (int c = 0; c < PER; ++c) acc[c] = acc[c] * f_old + v[c] * f_new;
     }
     const float inv = 1.f / ll;
-    const int i = row % K, sh = row / K, h = sh % H, s = sh / H;
-    __nv_bfloat16 *dst = out + ((static_cast<size_t>(s) * K + i) * H + h) * D + lane * PER;
+    const int h = hk * group + chunk * P.chunk_heads + r / P.K, i = r % P.K;
+    __nv_bfloat16 *dst = P.out + ((static_cast<size_t>(s) * P.K + i) * P.H + h) * D + lane * PER;
 #pragma unroll
     for (int c = 0; c < PER; c += 2)
         *reinterpret_cast<__nv_bfloat162 *>(dst + c) = __floats2bfloat162_rn(acc[c] * inv, acc[c + 1] * inv);
 }
 
 struct AttnPlan {
-    int chunk_heads, chunks, nsplit, items;
+    int chunk_heads, chunks, items, rows_per_item, tiles_per_item, workers, grid;
+    long long total_tiles;
+    bool any_cut;  // some item's tiles are spread over more than one share: partials + merge kernel needed
 };
 
 // Launch shape from host-known sizes only, so that the workspace query and the launch agree.
-AttnPlan make_plan(int S, int K, int H, int H_kv, int D, int max_prefix_len, int sm_count)
+AttnPlan make_plan(int S, int K, int H, int H_kv, int D, int max_prefix_len)
 {
     AttnPlan pl;
     const int group = H / H_kv;
     pl.chunk_heads = group < 16 / K ? group : 16 / K;
     if (pl.chunk_heads < 1) pl.chunk_heads = 1;
     pl.chunks = (group + pl.chunk_heads - 1) / pl.chunk_heads;
+    pl.rows_per_item = pl.chunk_heads * K;
     pl.items = S * H_kv * pl.chunks;
-    const int tiles = (max_prefix_len + K + kTileKeys - 1) / kTileKeys;
-    const int resident = sm_count * (D == 64 ? 3 : 2);  // blocks the GPU holds at once
-    int ns = (2 * resident + pl.items - 1) / pl.items;  // aim at two resident sets of blocks
-    const int max_by_len = tiles / 4 > 1 ? tiles / 4 : 1;  // at least four tiles per split
-    if (ns > max_by_len) ns = max_by_len;
-    if (ns < 1) ns = 1;
-    if (ns > 64) ns = 64;
-    pl.nsplit = ns;
+    const int tk = D == 64 ? AttnCfg<64>::kTileKeys : AttnCfg<128>::kTileKeys;
+    pl.tiles_per_item = (max_prefix_len + K + tk - 1) / tk;
+    pl.total_tiles = static_cast<long long>(pl.items) * pl.tiles_per_item;
+    const long long cap = static_cast<long long>(kPlanSms) * kWarps;
+    pl.workers = static_cast<int>(pl.total_tiles < cap ? pl.total_tiles : cap);
+    pl.grid = (pl.workers + kWarps - 1) / kWarps;
+    pl.any_cut = false;
+    for (int it = 0; it < pl.items && !pl.any_cut; ++it) {
+        const long long a = static_cast<long long>(it) * pl.tiles_per_item, b = a + pl.tiles_per_item;
+        pl.any_cut = owner(a, pl.total_tiles, pl.workers) != owner(b - 1, pl.total_tiles, pl.workers);
+    }
     return pl;
+}
+
+template <int D, int NQT>
+cudaError_t launch_attn(const CUtensorMap &map_k, const CUtensorMap &map_v, const AttnParams &P, int grid,
+                        cudaStream_t st)
+{
+    static bool attr_done = false;
+    if (!attr_done) {
+        const cudaError_t e = cudaFuncSetAttribute(attn_kernel<D, NQT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                   static_cast<int>(AttnCfg<D>::kSmemBytes));
+        if (e != cudaSuccess) return e;
+        attr_done = true;
+    }
+    return hawk_host::launch_dependent(attn_kernel<D, NQT>, dim3(grid), dim3(kThreads), AttnCfg<D>::kSmemBytes, st,
+                                       map_k, map_v, P);
 }
 
 }  // namespace
@@ -409,9 +605,9 @@ extern "C" size_t hawk_verify_attn_workspace_bytes(int S, int K, int H, int H_kv
     if (S <= 0 || K < 1 || K > 16 || H <= 0 || H_kv <= 0 || H % H_kv != 0 || (D != 64 && D != 128) ||
         max_prefix_len < 0)
         return 0;
-    const AttnPlan pl = make_plan(S, K, H, H_kv, D, max_prefix_len, 148);
-    if (pl.nsplit == 1) return 0;
-    return static_cast<size_t>(S) * H * K * pl.nsplit * (D + 2) * sizeof(float);
+    const AttnPlan pl = make_plan(S, K, H, H_kv, D, max_prefix_len);
+    if (!pl.any_cut) return 0;
+    return static_cast<size_t>(pl.workers) * 2 * 16 * (D + 2) * sizeof(float);
 }
 
 extern "C" hawk_status hawk_verify_attn(const void *q, const void *k_cache, const void *v_cache,
@@ -429,72 +625,59 @@ extern "C" hawk_status hawk_verify_attn(const void *q, const void *k_cache, cons
     if (!hawk_host::aligned16(q) || !hawk_host::aligned16(k_cache) || !hawk_host::aligned16(v_cache) ||
         !hawk_host::aligned16(out))
         return HAWK_ERR_ALIGN;
-    int sm_count = 0;
-    if (!hawk_host::is_sm100(&sm_count)) return HAWK_ERR_UNSUPPORTED;
-    (void)sm_count;  // the plan uses the B200's 148 SMs so that the workspace query needs no device
+    if (!hawk_host::is_sm100(nullptr)) return HAWK_ERR_UNSUPPORTED;
 
-    const AttnPlan pl = make_plan(S, K, H, H_kv, D, max_prefix_len, 148);
+    const AttnPlan pl = make_plan(S, K, H, H_kv, D, max_prefix_len);
     const size_t need = hawk_verify_attn_workspace_bytes(S, K, H, H_kv, D, max_prefix_len);
     if (need > 0) {
         if (!workspace || workspace_bytes < need) return HAWK_ERR_WORKSPACE;
         if (!hawk_host::aligned16(workspace)) return HAWK_ERR_ALIGN;
     }
 
+    const int tile_keys = D == 64 ? AttnCfg<64>::kTileKeys : AttnCfg<128>::kTileKeys;
     CUtensorMap map_k, map_v;
     const uint64_t rows = static_cast<uint64_t>(S) * H_kv * L_cap;
-    if (!hawk_host::encode_bf16_rows_sw128(&map_k, k_cache, rows, D, kTileKeys, true) ||
-        !hawk_host::encode_bf16_rows_sw128(&map_v, v_cache, rows, D, kTileKeys, true))
+    if (!hawk_host::encode_bf16_rows_sw128(&map_k, k_cache, rows, D, tile_keys, true) ||
+        !hawk_host::encode_bf16_rows_sw128(&map_v, v_cache, rows, D, tile_keys, true))
         return HAWK_ERR_CUDA;
 
     AttnParams P;
     P.q = static_cast<const __nv_bfloat16 *>(q);
     P.prefix_len = prefix_len;
     P.out = static_cast<__nv_bfloat16 *>(out);
-    P.part_o = static_cast<float *>(workspace);
-    P.part_ml = P.part_o ? P.part_o + static_cast<size_t>(S) * H * K * pl.nsplit * D : nullptr;
+    P.part = static_cast<float *>(workspace);
     P.S = S;
     P.K = K;
     P.H = H;
     P.H_kv = H_kv;
     P.L_cap = L_cap;
+    P.pl_max = max_prefix_len < L_cap - K ? max_prefix_len : L_cap - K;
     P.chunk_heads = pl.chunk_heads;
     P.chunks = pl.chunks;
-    P.nsplit = pl.nsplit;
+    P.tiles_per_item = pl.tiles_per_item;
+    P.workers = pl.workers;
+    P.total_tiles = pl.total_tiles;
     P.scale_log2 = sm_scale * 1.4426950408889634f;
     P.dev_status = dev_status;
 
     cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
-    const int grid = pl.items * pl.nsplit;
+    const bool wide = pl.rows_per_item > 8;  // more than one 8-query column tile
     cudaError_t err;
-    if (D == 64) {
-        static bool attr_done = false;
-        if (!attr_done) {
-            if (cudaFuncSetAttribute(attn_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                     static_cast<int>(AttnCfg<64>::kSmemBytes)) != cudaSuccess)
-                return HAWK_ERR_CUDA;
-            attr_done = true;
-        }
-        attn_kernel<64><<<grid, kThreads, AttnCfg<64>::kSmemBytes, st>>>(map_k, map_v, P);
-    } else {
-        static bool attr_done = false;
-        if (!attr_done) {
-            if (cudaFuncSetAttribute(attn_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                     static_cast<int>(AttnCfg<128>::kSmemBytes)) != cudaSuccess)
-                return HAWK_ERR_CUDA;
-            attr_done = true;
-        }
-        attn_kernel<128><<<grid, kThreads, AttnCfg<128>::kSmemBytes, st>>>(map_k, map_v, P);
-    }
-    err = cudaGetLastError();
+    if (D == 64)
+        err = wide ? launch_attn<64, 2>(map_k, map_v, P, pl.grid, st) : launch_attn<64, 1>(map_k, map_v, P, pl.grid, st);
+    else
+        err = wide ? launch_attn<128, 2>(map_k, map_v, P, pl.grid, st)
+                   : launch_attn<128, 1>(map_k, map_v, P, pl.grid, st);
     if (err != cudaSuccess) return HAWK_ERR_CUDA;
-    if (pl.nsplit > 1) {
-        const int rows_total = S * H * K;
-        const int threads = 256, blocks = (rows_total * 32 + threads - 1) / threads;
-        if (D == 64)
-            attn_combine_kernel<64><<<blocks, threads, 0, st>>>(P.part_o, P.part_ml, P.out, rows_total, K, H, pl.nsplit);
-        else
-            attn_combine_kernel<128><<<blocks, threads, 0, st>>>(P.part_o, P.part_ml, P.out, rows_total, K, H, pl.nsplit);
-        if (cudaGetLastError() != cudaSuccess) return HAWK_ERR_CUDA;
+    if (pl.any_cut) {
+        const int threads = 256;
+        const long long warps = static_cast<long long>(pl.items) * pl.rows_per_item;
+        const int blocks = static_cast<int>((warps * 32 + threads - 1) / threads);
+        err = D == 64 ? hawk_host::launch_dependent(attn_combine_kernel<64>, dim3(blocks), dim3(threads), 0, st, P,
+                                                    pl.items, pl.rows_per_item)
+                      : hawk_host::launch_dependent(attn_combine_kernel<128>, dim3(blocks), dim3(threads), 0, st, P,
+                                                    pl.items, pl.rows_per_item);
+        if (err != cudaSuccess) return HAWK_ERR_CUDA;
     }
     return HAWK_OK;
 }

@@ -39,6 +39,22 @@ __device__ __forceinline__ uint32_t elect_one()
     return pred;
 }
 
+// ---------------------------------------------------------------------------------- dependent launch
+// Every kernel of the library is launched with programmatic stream serialisation: it may be
+// scheduled while its predecessor in the stream still runs, does its set-up, and must call
+// grid_dependency_wait() before it touches global memory.  The wait returns once the predecessor has
+// completed and its writes are visible, so stream order is kept; what overlaps is launch latency and
+// set-up.  allow_dependent_launch() tells the scheduler that the next kernel may start that early.
+__device__ __forceinline__ void allow_dependent_launch()
+{
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+
+__device__ __forceinline__ void grid_dependency_wait()
+{
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+}
+
 // ---------------------------------------------------------------------------------- mbarrier
 __device__ __forceinline__ void mbar_init(uint64_t *bar, uint32_t count)
 {
@@ -300,5 +316,23 @@ bool encode_bf16_rows_sw128(CUtensorMap *map, const void *base, uint64_t rows, u
 bool is_sm100(int *sm_count);
 
 inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// Launches `kernel` with programmatic stream serialisation (see grid_dependency_wait()).
+template <class... KArgs, class... Args>
+inline cudaError_t launch_dependent(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream,
+                                    Args &&...args)
+{
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
 
 }  // namespace hawk_host

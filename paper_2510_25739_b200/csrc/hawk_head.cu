@@ -49,6 +49,7 @@ __global__ void __launch_bounds__(kHeadThreads, 1) head_proj_kernel(const __grid
     volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    hawk::allow_dependent_launch();
     const int kblocks = P.hidden / kBK;
     const int total_tiles = P.tiles_m * P.tiles_n;
 
@@ -72,6 +73,7 @@ __global__ void __launch_bounds__(kHeadThreads, 1) head_proj_kernel(const __grid
     __syncthreads();
     tcgen05_fence_after();
     const uint32_t tmem_base = *tmem_slot;
+    grid_dependency_wait();  // set-up above overlaps the previous kernel; global memory is touched from here on
 
     if (warp == 0) {
         // =========================== TMA producer
@@ -245,6 +247,7 @@ extern "C" hawk_status hawk_head_proj(const void *x, const void *w, float *logit
     }
     const int total_tiles = P.tiles_m * P.tiles_n;
     const int grid = total_tiles < sm_count ? total_tiles : sm_count;
-    head_proj_kernel<<<grid, kHeadThreads, smem_req, reinterpret_cast<cudaStream_t>(stream)>>>(map_w, map_x, P);
-    return cudaGetLastError() == cudaSuccess ? HAWK_OK : HAWK_ERR_CUDA;
+    const cudaError_t err = hawk_host::launch_dependent(head_proj_kernel, dim3(grid), dim3(kHeadThreads), smem_req,
+                                                        reinterpret_cast<cudaStream_t>(stream), map_w, map_x, P);
+    return err == cudaSuccess ? HAWK_OK : HAWK_ERR_CUDA;
 }

@@ -54,11 +54,13 @@ def test_step_struct_matches_the_header():
 
 
 def test_workspace_queries(lib):
-    # invalid shapes report 0; a split launch needs (D + 2) floats per (row, split)
+    # invalid shapes report 0; a launch that cuts items needs two 16-row fp32 partial slots per share
     assert lib.hawk_verify_attn_workspace_bytes(0, 4, 16, 16, 64, 128) == 0
     assert lib.hawk_verify_attn_workspace_bytes(2, 4, 16, 16, 96, 128) == 0
     need = lib.hawk_verify_attn_workspace_bytes(16, 5, 20, 20, 64, 1144)
-    assert need % (16 * 20 * 5 * 66 * 4) == 0
+    assert need > 0 and need % (2 * 16 * 66 * 4) == 0
+    # one tile per item and one share per tile: nothing is cut, no workspace
+    assert lib.hawk_verify_attn_workspace_bytes(2, 1, 1, 1, 64, 0) == 0
     assert lib.hawk_cfg_accept_workspace_bytes(8, 5, 16384) >= 8 * 5 * 4
     assert lib.hawk_cfg_accept_workspace_bytes(0, 5, 16384) == 0
 
