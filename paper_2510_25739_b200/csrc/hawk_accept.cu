@@ -1,10 +1,16 @@
 // hawk_cfg_accept: guidance combine, temperature, top-k, softmax, acceptance test and residual
-// resampling, one thread block per (sequence, draft position) row.
+// resampling.
 //
-// The row of guided logits lives in registers from the moment it is read (each logit row is read
-// from HBM exactly once); the target probabilities p and the residual max(0, p - q) are never
-// written back.  Draft probabilities q are read only by rows whose draft was rejected.
-// A second, tiny kernel picks, per sequence, the first rejected row.
+// One thread block per (sequence, draft position) row.  The row of guided logits lives in registers
+// from the moment it is read (each logit row is read from HBM exactly once); the target
+// probabilities p and the residual max(0, p - q) are never written back.  Draft probabilities q are
+// read only by rows whose draft was rejected.  A second, tiny kernel picks, per sequence, the first
+// rejected row.
+// The kernel is a chain of short block-wide phases (range, histogram select, softmax sum, scan), so
+// what bounds it is the length of that chain: the block is as wide as the row allows (16 ids per
+// thread, up to 1024 threads) and every phase is a handful of instructions per thread.
+// (Splitting a row over a cluster of blocks was measured: each cluster-wide exchange costs about
+// 1.2 us, five of them per row cost more than the wider load path saves.)
 //
 // Rule implemented: accept draft x iff u * q(x) < p(x); at the first rejection draw the
 // correction token from norm(max(0, p - q)) by inverse CDF in ascending token id
@@ -17,9 +23,9 @@
 
 namespace {
 
-constexpr int kBins = 2048;     // histogram bins of one top-k selection round
-constexpr int kCandMax = 2048;  // candidates ranked exactly in shared memory
-constexpr int kMaxRounds = 48;  // each round shrinks the value range by >= 2048x; fp32 allows < 16
+constexpr int kBins = 1024;     // histogram bins of one top-k selection round
+constexpr int kCandMax = 1024;  // members of the selected bin that are ranked exactly in shared memory
+constexpr int kMaxRounds = 48;  // each narrowing round shrinks the value range by >= 1024x; fp32 allows < 8
 
 constexpr int ROW_ACCEPTED = -1;
 constexpr int ROW_REJECTED_NO_TOKEN = -2;  // rejected and nothing has positive mass
@@ -57,74 +63,80 @@ __device__ __forceinline__ float4 load4(const float *row, int e, int n, bool vec
     return r;
 }
 
-// Guided logit in fp32: subtract, fused multiply-add, divide (three correctly rounded steps).
-__device__ __forceinline__ float guided(float c, float u, float s, float T, int &flags)
+// Guided logit in fp32: subtract, fused multiply-add, divide (three correctly rounded steps; a
+// temperature of exactly 1 leaves the value as it is, so the divide is skipped).
+// -inf in either stream gives -inf; NaN or +inf anywhere (inputs or result) gives -inf and a flag.
+__device__ __forceinline__ float guided(float c, float u, float s, float T, bool unit_T, int &flags)
 {
-    const bool bad_c = (c != c) || c == CUDART_INF_F, bad_u = (u != u) || u == CUDART_INF_F;
-    if (bad_c || bad_u) flags |= HAWK_DEV_NONFINITE;
-    if (bad_c || bad_u || c == -CUDART_INF_F || u == -CUDART_INF_F) return -CUDART_INF_F;
-    float r = __fdiv_rn(__fmaf_rn(s, __fsub_rn(c, u), u), T);
-    if ((r != r) || r == CUDART_INF_F) {
-        flags |= HAWK_DEV_NONFINITE;
-        r = -CUDART_INF_F;
+    if (fabsf(c) < CUDART_INF_F && fabsf(u) < CUDART_INF_F) {  // both finite: the common case
+        float r = __fmaf_rn(s, __fsub_rn(c, u), u);
+        if (!unit_T) r = __fdiv_rn(r, T);
+        if (fabsf(r) < CUDART_INF_F) return r;
+        if (r != -CUDART_INF_F) flags |= HAWK_DEV_NONFINITE;  // overflow to +inf or NaN
+        return -CUDART_INF_F;
     }
-    return r;
+    if ((c != c) || (u != u) || c == CUDART_INF_F || u == CUDART_INF_F) flags |= HAWK_DEV_NONFINITE;
+    return -CUDART_INF_F;
 }
+
+// Order-preserving map between fp32 values (no NaN) and int32; it is its own inverse.
+__device__ __forceinline__ int ordered_int(float v)
+{
+    const int k = __float_as_int(v);
+    return k ^ ((k >> 31) & 0x7fffffff);
+}
+__device__ __forceinline__ float ordered_float(int k) { return __int_as_float(k ^ ((k >> 31) & 0x7fffffff)); }
 
 template <int NT>
 struct Scratch {
     float f[3][32];
-    int i[32];
+    int i[32], i2[32], i3[32];
     float scan[33];
+    int iscan[33];
 };
 
+// Block-wide max, min and count: one redux instruction per value and level instead of shuffle trees.
 template <int NT>
 __device__ __forceinline__ void block_minmaxcount(float &mx, float &mn, int &cnt, Scratch<NT> &s)
 {
-    constexpr int NW = NT / 32;
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
-        mn = fminf(mn, __shfl_xor_sync(0xffffffffu, mn, o));
-        cnt += __shfl_xor_sync(0xffffffffu, cnt, o);
-    }
+    constexpr int kNW = NT / 32;
+    int kmx = __reduce_max_sync(0xffffffffu, ordered_int(mx));
+    int kmn = __reduce_min_sync(0xffffffffu, ordered_int(mn));
+    cnt = __reduce_add_sync(0xffffffffu, cnt);
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     __syncthreads();
     if (lane == 0) {
-        s.f[0][warp] = mx;
-        s.f[1][warp] = mn;
-        s.i[warp] = cnt;
+        s.i[warp] = kmx;
+        s.i2[warp] = kmn;
+        s.i3[warp] = cnt;
     }
     __syncthreads();
-    mx = lane < NW ? s.f[0][lane] : -CUDART_INF_F;
-    mn = lane < NW ? s.f[1][lane] : CUDART_INF_F;
-    cnt = lane < NW ? s.i[lane] : 0;
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
-        mn = fminf(mn, __shfl_xor_sync(0xffffffffu, mn, o));
-        cnt += __shfl_xor_sync(0xffffffffu, cnt, o);
-    }
+    kmx = __reduce_max_sync(0xffffffffu, lane < kNW ? s.i[lane] : ordered_int(-CUDART_INF_F));
+    kmn = __reduce_min_sync(0xffffffffu, lane < kNW ? s.i2[lane] : ordered_int(CUDART_INF_F));
+    cnt = __reduce_add_sync(0xffffffffu, lane < kNW ? s.i3[lane] : 0);
+    mx = ordered_float(kmx);
+    mn = ordered_float(kmn);
 }
 
 template <int NT>
 __device__ __forceinline__ float block_sum(float v, Scratch<NT> &s)
 {
-    constexpr int NW = NT / 32;
+    constexpr int kNW = NT / 32;
     v = hawk::warp_sum(v);
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     __syncthreads();
     if (lane == 0) s.f[0][warp] = v;
     __syncthreads();
-    v = lane < NW ? s.f[0][lane] : 0.f;
+    v = lane < kNW ? s.f[0][lane] : 0.f;
     return hawk::warp_sum(v);
 }
 
-// Exclusive prefix sum over the block in thread order; *total receives the block sum.
+// Exclusive prefix sum over the block in thread order; *total receives the block sum.  Two barriers:
+// the warp totals go through shared memory once and every warp scans them for itself.
 template <int NT, class T>
-__device__ __forceinline__ T block_exclusive_scan(T v, T *scratch33, T *total)
+__device__ __forceinline__ T block_exclusive_scan(T v, T *scratch32, T *total)
 {
-    constexpr int NW = NT / 32;
+    constexpr int kNW = NT / 32;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     T incl = v;
 #pragma unroll
@@ -132,25 +144,21 @@ __device__ __forceinline__ T block_exclusive_scan(T v, T *scratch33, T *total)
         T up = __shfl_up_sync(0xffffffffu, incl, o);
         if (lane >= o) incl += up;
     }
+    __syncthreads();  // earlier readers of scratch32 are done
+    if (lane == 31) scratch32[warp] = incl;
     __syncthreads();
-    if (lane == 31) scratch33[warp] = incl;
-    __syncthreads();
-    if (warp == 0) {
-        T w = lane < NW ? scratch33[lane] : T(0);
-        T wi = w;
+    const T w = lane < kNW ? scratch32[lane] : T(0);
+    T wi = w;
 #pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-            T up = __shfl_up_sync(0xffffffffu, wi, o);
-            if (lane >= o) wi += up;
-        }
-        scratch33[lane] = wi - w;
-        if (lane == 31) scratch33[32] = wi;
+    for (int o = 1; o < 32; o <<= 1) {
+        T up = __shfl_up_sync(0xffffffffu, wi, o);
+        if (lane >= o) wi += up;
     }
-    __syncthreads();
-    *total = scratch33[32];
-    return scratch33[warp] + (incl - v);
+    *total = __shfl_sync(0xffffffffu, wi, 31);
+    return __shfl_sync(0xffffffffu, wi - w, warp) + (incl - v);
 }
 
+// NT threads, VPT float4 loads per thread: the block holds up to 4 * NT * VPT valid ids of its row.
 template <int NT, int VPT>
 __global__ void __launch_bounds__(NT) accept_rows_kernel(const AcceptParams P)
 {
@@ -162,15 +170,15 @@ __global__ void __launch_bounds__(NT) accept_rows_kernel(const AcceptParams P)
     __shared__ int s_hist[kBins];
     __shared__ float s_cand[kCandMax];
     __shared__ Scratch<NT> s_red;
-    __shared__ int s_iscan[33];
     __shared__ float s_wt[VPT * NW];
     __shared__ float s_wbase[VPT * NW];
-    __shared__ int s_ncand, s_bin, s_above, s_tok;
-    __shared__ float s_tau, s_px;
+    __shared__ int s_bin, s_above, s_tok;
+    __shared__ float s_tau, s_pxe, s_total;
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     hawk::allow_dependent_launch();
     hawk::grid_dependency_wait();
+
     const int row = blockIdx.x;  // position-major: all rows of position 0 first
     const int i = row / P.B, b = row - i * P.B;
     const bool bonus = (i == P.K);
@@ -181,7 +189,38 @@ __global__ void __launch_bounds__(NT) accept_rows_kernel(const AcceptParams P)
     const float *qrow = bonus ? nullptr : P.q + (static_cast<size_t>(b) * P.K + i) * P.V + P.v_begin;
     int flags = 0;
 
-    // draft id, its q and the uniforms: issued early so the latency hides behind the row load
+    const bool unit_T = P.temperature == 1.0f;
+    // ---- read both logit rows once, combine into registers
+    float x[VPT][4];
+    float mx = -CUDART_INF_F, mn = CUDART_INF_F;
+    int cnt = 0;
+    {
+        float4 c4[VPT], u4[VPT];
+#pragma unroll
+        for (int j = 0; j < VPT; ++j) {  // all loads in flight before the first use
+            const int e0 = 4 * (j * NT + tid);
+            c4[j] = e0 < n ? load4(lc, e0, n, vec_ok, -CUDART_INF_F) : make_float4(0.f, 0.f, 0.f, 0.f);
+            u4[j] = e0 < n ? load4(lu, e0, n, vec_ok, -CUDART_INF_F) : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+#pragma unroll
+        for (int j = 0; j < VPT; ++j) {
+            const int e0 = 4 * (j * NT + tid);
+            int fl = 0;
+            x[j][0] = e0 + 0 < n ? guided(c4[j].x, u4[j].x, P.cfg_scale, P.temperature, unit_T, fl) : -CUDART_INF_F;
+            x[j][1] = e0 + 1 < n ? guided(c4[j].y, u4[j].y, P.cfg_scale, P.temperature, unit_T, fl) : -CUDART_INF_F;
+            x[j][2] = e0 + 2 < n ? guided(c4[j].z, u4[j].z, P.cfg_scale, P.temperature, unit_T, fl) : -CUDART_INF_F;
+            x[j][3] = e0 + 3 < n ? guided(c4[j].w, u4[j].w, P.cfg_scale, P.temperature, unit_T, fl) : -CUDART_INF_F;
+            flags |= fl;
+#pragma unroll
+            for (int c = 0; c < 4; ++c)
+                if (x[j][c] > -CUDART_INF_F) {
+                    mx = fmaxf(mx, x[j][c]);
+                    mn = fminf(mn, x[j][c]);
+                    ++cnt;
+                }
+        }
+    }
+    // draft id, its q and the uniforms
     int xd = 0;
     float qx = 0.f, u_acc = 0.f;
     if (!bonus) {
@@ -195,37 +234,9 @@ __global__ void __launch_bounds__(NT) accept_rows_kernel(const AcceptParams P)
         u_acc = P.u_acc[b * P.K + i];
     }
     const float u_res = P.u_res[b * (P.K + 1) + i];
-
-    // ---- read both logit rows once, combine into registers
-    float x[VPT][4];
-    float mx = -CUDART_INF_F, mn = CUDART_INF_F;
-    int cnt = 0;
-#pragma unroll
-    for (int j = 0; j < VPT; ++j) {
-        const int e0 = 4 * (j * NT + tid);
-        if (e0 < n) {
-            const float4 c4 = load4(lc, e0, n, vec_ok, -CUDART_INF_F);
-            const float4 u4 = load4(lu, e0, n, vec_ok, -CUDART_INF_F);
-            int fl = 0;
-            x[j][0] = guided(c4.x, u4.x, P.cfg_scale, P.temperature, fl);
-            x[j][1] = e0 + 1 < n ? guided(c4.y, u4.y, P.cfg_scale, P.temperature, fl) : -CUDART_INF_F;
-            x[j][2] = e0 + 2 < n ? guided(c4.z, u4.z, P.cfg_scale, P.temperature, fl) : -CUDART_INF_F;
-            x[j][3] = e0 + 3 < n ? guided(c4.w, u4.w, P.cfg_scale, P.temperature, fl) : -CUDART_INF_F;
-            flags |= fl;
-        } else {
-            x[j][0] = x[j][1] = x[j][2] = x[j][3] = -CUDART_INF_F;
-        }
-#pragma unroll
-        for (int c = 0; c < 4; ++c)
-            if (x[j][c] > -CUDART_INF_F) {
-                mx = fmaxf(mx, x[j][c]);
-                mn = fminf(mn, x[j][c]);
-                ++cnt;
-            }
-    }
-    block_minmaxcount<NT>(mx, mn, cnt, s_red);
-
     if (flags && P.dev_status) atomicOr(P.dev_status, flags);
+
+    block_minmaxcount<NT>(mx, mn, cnt, s_red);
 
     if (cnt == 0) {  // nothing has mass: p == 0 everywhere, the draft is rejected, no token exists
         if (P.p_debug) {
@@ -246,27 +257,28 @@ __global__ void __launch_bounds__(NT) accept_rows_kernel(const AcceptParams P)
                 tau = hi;
                 break;
             }
+            // histogram of the values in [lo, hi]: bin 0 holds the largest
             const float scale = static_cast<float>(kBins) / (hi - lo);
-            for (int t = tid; t < kBins; t += NT) s_hist[t] = 0;
-            if (tid == 0) s_ncand = 0;
+#pragma unroll
+            for (int t = 0; t < BPT; ++t) s_hist[t * NT + tid] = 0;
             __syncthreads();
+            int bins[VPT][4];  // bin of every value held (-1: outside [lo, hi])
 #pragma unroll
             for (int j = 0; j < VPT; ++j)
 #pragma unroll
                 for (int c = 0; c < 4; ++c) {
                     const float v = x[j][c];
-                    if (v >= lo && v <= hi) {
-                        const int bin = min(kBins - 1, static_cast<int>((hi - v) * scale));
-                        atomicAdd(&s_hist[bin], 1);
-                    }
+                    const bool in = v >= lo && v <= hi;
+                    bins[j][c] = in ? min(kBins - 1, static_cast<int>((hi - v) * scale)) : -1;
+                    if (in) atomicAdd(&s_hist[bins[j][c]], 1);
                 }
             __syncthreads();
             int local = 0;
 #pragma unroll
             for (int t = 0; t < BPT; ++t) local += s_hist[tid * BPT + t];
             int total;
-            const int excl = block_exclusive_scan<NT, int>(local, s_iscan, &total);
-            if (excl < k && k <= excl + local) {
+            const int excl = block_exclusive_scan<NT, int>(local, s_red.iscan, &total);
+            if (excl < k && k <= excl + local) {  // exactly one thread: one of its bins holds the k-th largest
                 int run = excl;
 #pragma unroll
                 for (int t = 0; t < BPT; ++t) {
@@ -281,47 +293,62 @@ __global__ void __launch_bounds__(NT) accept_rows_kernel(const AcceptParams P)
             __syncthreads();
             const int bstar = s_bin, kk = k - s_above, C = s_hist[bstar];
             if (C <= kCandMax) {
+                // rank the members of the bin exactly: the kk-th largest of them is the threshold.
+                // They are compacted into shared memory by a prefix sum over the threads' member counts
+                // (atomics on one counter would serialise).
+                int mine = 0;
 #pragma unroll
                 for (int j = 0; j < VPT; ++j)
 #pragma unroll
-                    for (int c = 0; c < 4; ++c) {
-                        const float v = x[j][c];
-                        if (v >= lo && v <= hi) {
-                            const int bin = min(kBins - 1, static_cast<int>((hi - v) * scale));
-                            if (bin == bstar) s_cand[atomicAdd(&s_ncand, 1)] = v;
-                        }
-                    }
+                    for (int c = 0; c < 4; ++c) mine += bins[j][c] == bstar;
+                int ctotal;
+                int pos = block_exclusive_scan<NT, int>(mine, s_red.iscan, &ctotal);
+                if (mine) {
+#pragma unroll
+                    for (int j = 0; j < VPT; ++j)
+#pragma unroll
+                        for (int c = 0; c < 4; ++c)
+                            if (bins[j][c] == bstar) s_cand[pos++] = x[j][c];
+                }
                 __syncthreads();
-                for (int t = tid; t < C; t += NT) {
-                    const float v = s_cand[t];
-                    int gt = 0, ge = 0;
-                    for (int m = 0; m < C; ++m) {
-                        const float w = s_cand[m];
-                        gt += w > v;
-                        ge += w >= v;
+                if (C <= 32) {  // the usual case: one warp ranks them with shuffles
+                    if (warp == 0) {
+                        const float v = lane < C ? s_cand[lane] : -CUDART_INF_F;
+                        int gt = 0, ge = 0;
+                        for (int m = 0; m < C; ++m) {
+                            const float w = __shfl_sync(0xffffffffu, v, m);
+                            gt += w > v;
+                            ge += w >= v;
+                        }
+                        if (lane < C && gt < kk && kk <= ge) s_tau = v;
                     }
-                    if (gt < kk && kk <= ge) s_tau = v;
+                } else {
+                    for (int t = tid; t < C; t += NT) {
+                        const float v = s_cand[t];
+                        int gt = 0, ge = 0;
+                        for (int m = 0; m < C; ++m) {
+                            const float w = s_cand[m];
+                            gt += w > v;
+                            ge += w >= v;
+                        }
+                        if (gt < kk && kk <= ge) s_tau = v;  // several threads may hold the same value
+                    }
                 }
                 __syncthreads();
                 tau = s_tau;
                 break;
             }
-            // too many candidates share the bin: narrow the range to that bin's values and repeat
+            // too many members share the bin: narrow the range to their values and repeat
             float nmx = -CUDART_INF_F, nmn = CUDART_INF_F;
             int dummy = 0;
 #pragma unroll
             for (int j = 0; j < VPT; ++j)
 #pragma unroll
-                for (int c = 0; c < 4; ++c) {
-                    const float v = x[j][c];
-                    if (v >= lo && v <= hi) {
-                        const int bin = min(kBins - 1, static_cast<int>((hi - v) * scale));
-                        if (bin == bstar) {
-                            nmx = fmaxf(nmx, v);
-                            nmn = fminf(nmn, v);
-                        }
+                for (int c = 0; c < 4; ++c)
+                    if (bins[j][c] == bstar) {
+                        nmx = fmaxf(nmx, x[j][c]);
+                        nmn = fminf(nmn, x[j][c]);
                     }
-                }
             block_minmaxcount<NT>(nmx, nmn, dummy, s_red);
             lo = nmn;
             hi = nmx;
@@ -337,12 +364,20 @@ __global__ void __launch_bounds__(NT) accept_rows_kernel(const AcceptParams P)
     for (int j = 0; j < VPT; ++j)
 #pragma unroll
         for (int c = 0; c < 4; ++c) {
-            const float v = x[j][c];
-            const float e = (v >= tau && v > -CUDART_INF_F) ? hawk::fast_exp2((v - mx) * kLog2e) : 0.f;
+            const float v = x[j][c];  // -inf gives exp2(-inf) = 0
+            const float e = v >= tau ? hawk::fast_exp2((v - mx) * kLog2e) : 0.f;
             x[j][c] = e;
             zsum += e;
         }
+    if (!bonus && tid == ((xd >> 2) % NT)) {  // the thread that holds the draft id
+#pragma unroll
+        for (int j = 0; j < VPT; ++j)
+#pragma unroll
+            for (int c = 0; c < 4; ++c)
+                if (4 * (j * NT + tid) + c == xd) s_pxe = x[j][c];
+    }
     const float Z = block_sum<NT>(zsum, s_red);
+    const float pxe = s_pxe;
     const float invZ = 1.0f / Z;
 
     if (P.p_debug) {
@@ -356,15 +391,9 @@ __global__ void __launch_bounds__(NT) accept_rows_kernel(const AcceptParams P)
             }
     }
 
-    // ---- acceptance test on the draft token
+    // ---- acceptance test on the draft token 
     if (!bonus) {
-#pragma unroll
-        for (int j = 0; j < VPT; ++j)
-#pragma unroll
-            for (int c = 0; c < 4; ++c)
-                if (4 * (j * NT + tid) + c == xd) s_px = x[j][c] * invZ;
-        __syncthreads();
-        const float px = s_px;
+        const float px = pxe * invZ;
         const bool accepted = static_cast<double>(u_acc) * static_cast<double>(qx) < static_cast<double>(px);
         if (accepted) {
             if (tid == 0) P.row_out[b * P.rows + i] = ROW_ACCEPTED;
@@ -375,15 +404,22 @@ __global__ void __launch_bounds__(NT) accept_rows_kernel(const AcceptParams P)
     // ---- rejected (or bonus row): inverse-CDF draw from max(0, p - q), or from p itself
     bool use_q = !bonus;
     for (int attempt = 0; attempt < 2; ++attempt) {
-        float sj[VPT];
+        float rr[VPT][4], sj[VPT];  // residual weights of this thread's ids and their sums per group of 4
+        {
+            float4 q4[VPT];
 #pragma unroll
-        for (int j = 0; j < VPT; ++j) {
-            const int e0 = 4 * (j * NT + tid);
-            float4 q4 = make_float4(0.f, 0.f, 0.f, 0.f);
-            if (use_q && e0 < n) q4 = load4(qrow, e0, n, vec_ok, 0.f);
-            const float r0 = fmaxf(0.f, x[j][0] * invZ - q4.x), r1 = fmaxf(0.f, x[j][1] * invZ - q4.y);
-            const float r2 = fmaxf(0.f, x[j][2] * invZ - q4.z), r3 = fmaxf(0.f, x[j][3] * invZ - q4.w);
-            sj[j] = ((r0 + r1) + r2) + r3;
+            for (int j = 0; j < VPT; ++j) {  // all loads in flight before the first use
+                const int e0 = 4 * (j * NT + tid);
+                q4[j] = (use_q && e0 < n) ? load4(qrow, e0, n, vec_ok, 0.f) : make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+#pragma unroll
+            for (int j = 0; j < VPT; ++j) {
+                rr[j][0] = fmaxf(0.f, x[j][0] * invZ - q4[j].x);
+                rr[j][1] = fmaxf(0.f, x[j][1] * invZ - q4[j].y);
+                rr[j][2] = fmaxf(0.f, x[j][2] * invZ - q4[j].z);
+                rr[j][3] = fmaxf(0.f, x[j][3] * invZ - q4[j].w);
+                sj[j] = ((rr[j][0] + rr[j][1]) + rr[j][2]) + rr[j][3];
+            }
         }
         float incl[VPT];
 #pragma unroll
@@ -398,39 +434,53 @@ __global__ void __launch_bounds__(NT) accept_rows_kernel(const AcceptParams P)
             if (lane == 31) s_wt[j * NW + warp] = v;
         }
         __syncthreads();
-        float total;
-        {
-            const float v = tid < VPT * NW ? s_wt[tid] : 0.f;
-            const float ex = block_exclusive_scan<NT, float>(v, s_red.scan, &total);
-            if (tid < VPT * NW) s_wbase[tid] = ex;
-            if (tid == 0) s_tok = 0x7fffffff;
+        if (warp == 0) {  // exclusive prefix of the VPT * NW warp totals (ascending id order), by one warp
+            constexpr int E = VPT * NW, PER = (E + 31) / 32;
+            float ent[PER], run = 0.f;
+#pragma unroll
+            for (int t = 0; t < PER; ++t) {
+                ent[t] = lane * PER + t < E ? s_wt[lane * PER + t] : 0.f;
+                run += ent[t];
+            }
+            float incl_l = run;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const float up = __shfl_up_sync(0xffffffffu, incl_l, o);
+                if (lane >= o) incl_l += up;
+            }
+            float base = incl_l - run;
+#pragma unroll
+            for (int t = 0; t < PER; ++t) {
+                if (lane * PER + t < E) s_wbase[lane * PER + t] = base;
+                base += ent[t];
+            }
+            if (lane == 31) s_total = incl_l;
+            if (lane == 0) s_tok = 0x7fffffff;
         }
         __syncthreads();
+        const float total = s_total;
         if (use_q && !(total > 0.f)) {  // p <= q everywhere: draw from p with the same uniform
             use_q = false;
             continue;
         }
-        const float t = u_res * total;
-        // pass 0: elements where the running sum crosses t; pass 1 (only if the block-wide sums
-        // disagree at a thread boundary): the first element whose running sum exceeds t
+        const float tl = u_res * total;
+        // pass 0: elements where the running sum crosses tl; pass 1 (only if the block-wide sums
+        // disagree at a thread boundary): the first element whose running sum exceeds tl
         for (int pass = 0; pass < 2; ++pass) {
 #pragma unroll
             for (int j = 0; j < VPT; ++j) {
                 const float excl = s_wbase[j * NW + warp] + (incl[j] - sj[j]);
-                const bool look = pass == 0 ? (excl <= t && excl + sj[j] > t) : (excl + sj[j] > t);
+                const bool look = pass == 0 ? (excl <= tl && excl + sj[j] > tl) : (excl + sj[j] > tl);
                 if (look) {
                     const int e0 = 4 * (j * NT + tid);
-                    float4 q4 = make_float4(0.f, 0.f, 0.f, 0.f);
-                    if (use_q && e0 < n) q4 = load4(qrow, e0, n, vec_ok, 0.f);
-                    const float r0 = fmaxf(0.f, x[j][0] * invZ - q4.x), r1 = fmaxf(0.f, x[j][1] * invZ - q4.y);
-                    const float r2 = fmaxf(0.f, x[j][2] * invZ - q4.z), r3 = fmaxf(0.f, x[j][3] * invZ - q4.w);
+                    const float r0 = rr[j][0], r1 = rr[j][1], r2 = rr[j][2], r3 = rr[j][3];
                     const float c0 = excl + r0, c1 = excl + (r0 + r1), c2 = excl + ((r0 + r1) + r2);
                     const float c3 = excl + (((r0 + r1) + r2) + r3);
                     int hit = -1;  // an id without mass is never drawn
-                    if (r0 > 0.f && c0 > t) hit = 0;
-                    else if (r1 > 0.f && c1 > t) hit = 1;
-                    else if (r2 > 0.f && c2 > t) hit = 2;
-                    else if (r3 > 0.f && c3 > t) hit = 3;
+                    if (r0 > 0.f && c0 > tl) hit = 0;
+                    else if (r1 > 0.f && c1 > tl) hit = 1;
+                    else if (r2 > 0.f && c2 > tl) hit = 2;
+                    else if (r3 > 0.f && c3 > tl) hit = 3;
                     if (hit >= 0) atomicMin(&s_tok, e0 + hit);
                 }
             }
@@ -439,7 +489,7 @@ __global__ void __launch_bounds__(NT) accept_rows_kernel(const AcceptParams P)
             __syncthreads();
         }
         int tok = s_tok;
-        if (tok == 0x7fffffff) {  // rounding left no running sum above t: the last id with mass
+        if (tok == 0x7fffffff) {  // rounding left no running sum above tl: the last id with mass
             __syncthreads();
             if (tid == 0) s_tok = -1;
             __syncthreads();
@@ -447,14 +497,10 @@ __global__ void __launch_bounds__(NT) accept_rows_kernel(const AcceptParams P)
             for (int j = 0; j < VPT; ++j) {
                 const int e0 = 4 * (j * NT + tid);
                 if (sj[j] > 0.f) {
-                    float4 q4 = make_float4(0.f, 0.f, 0.f, 0.f);
-                    if (use_q && e0 < n) q4 = load4(qrow, e0, n, vec_ok, 0.f);
-                    const float r[4] = {x[j][0] * invZ - q4.x, x[j][1] * invZ - q4.y, x[j][2] * invZ - q4.z,
-                                        x[j][3] * invZ - q4.w};
                     int last = -1;
 #pragma unroll
                     for (int c = 0; c < 4; ++c)
-                        if (r[c] > 0.f) last = e0 + c;
+                        if (rr[j][c] > 0.f) last = e0 + c;
                     if (last >= 0) atomicMax(&s_tok, last);
                 }
             }
@@ -490,6 +536,7 @@ __global__ void accept_finalize_kernel(const int32_t *row_out, int B, int K, int
     accept_len[b] = len;
     out_token[b] = tok;
 }
+
 
 template <int NT, int VPT>
 cudaError_t launch_rows(const AcceptParams &P, int grid, cudaStream_t stream)
@@ -552,11 +599,10 @@ extern "C" hawk_status hawk_cfg_accept(const float *logits, const float *q_probs
 
     cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
     const int grid = B * P.rows;
-    cudaError_t err;
-    if (n <= 1024) err = launch_rows<128, 2>(P, grid, st);
-    else if (n <= 4096) err = launch_rows<256, 4>(P, grid, st);
+    cudaError_t err;  // 16 ids per thread; the block as wide as the row needs
+    if (n <= 4096) err = launch_rows<256, 4>(P, grid, st);
     else if (n <= 8192) err = launch_rows<512, 4>(P, grid, st);
-    else if (n <= 16384) err = launch_rows<512, 8>(P, grid, st);
+    else if (n <= 16384) err = launch_rows<1024, 4>(P, grid, st);
     else err = launch_rows<1024, 8>(P, grid, st);
     if (err != cudaSuccess) return HAWK_ERR_CUDA;
     err = hawk_host::launch_dependent(accept_finalize_kernel, dim3((B + 127) / 128), dim3(128), 0, st,
