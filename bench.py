@@ -42,6 +42,12 @@ UNIT = "positions/s"
 L2_BYTES = 126 * 1024 * 1024
 
 
+# DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) of one hawk_verify_attn call, attention kernel
+# plus merge kernel, from the ncu capture summarised in profiles/; None where no capture of the
+# current kernels exists for that workload.
+ATTN_TRAFFIC_BYTES = {2: None}
+
+
 def measured_peaks():
     p = ROOT / "MEASURED_PEAKS.json"
     if p.exists():
@@ -405,7 +411,7 @@ def main():
     achieved = attn_bytes(cfg) / attn_s / 1e9
     roofline = {"kernel": "hawk_verify_attn", "bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"],
                 "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"], "peak_source": f"of {peaks['source']}",
-                "traffic": None, "us_per_launch": attn_s * 1e6, "algorithmic_bytes": attn_bytes(cfg),
+                "traffic": ATTN_TRAFFIC_BYTES.get(cid), "us_per_launch": attn_s * 1e6, "algorithmic_bytes": attn_bytes(cfg),
                 "timing": timing_mode}
 
     # ---- per-kernel loops (each kernel alone, rotating replicas) for the stage breakdown
@@ -451,8 +457,9 @@ def main():
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K_steps, "warmup": W,
         "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": "bf16 (attention, head operands) / f32 (accumulation, logits, accept)", "data": "synthetic",
+        "dtype": "bf16", "data": "synthetic",
         "config": {"workload": workload_name(cfg, cid), "positions_per_step_per_gpu": positions,
+                   "arithmetic": "bf16 operands (Q, K, V, X, W), fp32 accumulation, fp32 logits and accept stage",
                    "l2": f"inputs rotate over {n_rep} replicas ({n_rep * first.bytes() / 1e6:.0f} MB > 3x L2)",
                    "launch": "one CUDA graph replay per step (3 C-ABI calls captured)",
                    "parallelism": f"{world} independent replicas, sequences sharded, no collective"},
@@ -461,7 +468,7 @@ def main():
     }
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         _, t1, _ = oracle_sample(cfg, wl.seed_for(cid), 1)
-        reps_cpu = max(1, min(500, int(12.0 / max(t1, 1e-3))))     # about 10-15 s of CPU work
+        reps_cpu = max(1, min(2000, int(15.0 / max(t1, 1e-3))))    # about 15 s of CPU work
         v, dt, cores = oracle_sample(cfg, wl.seed_for(cid), reps_cpu)
         line["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle",
                                 "sample": f"{reps_cpu} full steps of the workload ({dt:.1f} s)"}

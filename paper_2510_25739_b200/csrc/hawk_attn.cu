@@ -487,63 +487,96 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const __grid_constant
 }
 
 // Merges the partial results of every item whose tiles were spread over several shares:
-// one warp per (item, query row of the item), lanes across the head dimension.
+// one warp per (item, query row of the item), lanes across the head dimension.  All index
+// arithmetic comes before the wait on the attention kernel; after it the loads of up to kAhead
+// contributions are issued together, so the kernel adds one memory round trip to the call.
 template <int D>
 __global__ void attn_combine_kernel(const AttnParams P, int items, int rows_per_item)
 {
     constexpr int TK = AttnCfg<D>::kTileKeys;
+    constexpr int PER = D / 32;
+    constexpr int kAhead = 4;
     allow_dependent_launch();
-    grid_dependency_wait();  // every thread waits, so this grid cannot retire before the attention kernel has
     const int wid = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const int lane = threadIdx.x & 31;
     const int item = wid / rows_per_item, r = wid - item * rows_per_item;
-    if (item >= items) return;
     const long long T = P.total_tiles;
     const long long a = static_cast<long long>(item) * P.tiles_per_item, b = a + P.tiles_per_item;
-    const int g_first = owner(a, T, P.workers), g_last = owner(b - 1, T, P.workers);
-    if (g_first == g_last) return;  // one share held the whole item and wrote the result itself
-    int it = item;
-    const int chunk = it % P.chunks;
-    it /= P.chunks;
-    const int hk = it % P.H_kv, s = it / P.H_kv;
+    bool active = item < items;
+    int g_first = 0, g_last = 0, s = 0, hk = 0, chunk = 0;
     const int group = P.H / P.H_kv;
-    const int nheads = min(P.chunk_heads, group - chunk * P.chunk_heads);
-    if (r >= nheads * P.K) return;
-    const int pl = max(0, min(P.prefix_len[s], P.pl_max));
-    const int ntiles = (pl + P.K + TK - 1) / TK;
+    if (active) {
+        g_first = owner(a, T, P.workers);
+        g_last = owner(b - 1, T, P.workers);
+        int it = item;
+        chunk = it % P.chunks;
+        it /= P.chunks;
+        hk = it % P.H_kv;
+        s = it / P.H_kv;
+        const int nheads = min(P.chunk_heads, group - chunk * P.chunk_heads);
+        // one share held the whole item and wrote the result itself; rows past the item's last do not exist
+        active = g_first != g_last && r < nheads * P.K;
+    }
+    // tile offset inside the item at which each contribution starts, and where it is stored
+    const float *slot[kAhead];
+    int seg_off[kAhead];
+#pragma unroll
+    for (int t = 0; t < kAhead; ++t) {
+        const int gg = min(g_first + t, g_last);
+        const long long sb = share_begin(gg, T, P.workers);
+        seg_off[t] = static_cast<int>((sb > a ? sb : a) - a);
+        slot[t] = P.part + (static_cast<size_t>(gg) * 2 + (a <= sb ? 0 : 1)) * 16 * (D + 2);
+    }
+    grid_dependency_wait();  // every thread waits, so this grid cannot retire before the attention kernel has
+    if (!active) return;
 
-    constexpr int PER = D / 32;
+    float2 ml[kAhead];
+    float v[kAhead][PER];
+    const int pl_raw = P.prefix_len[s];
+#pragma unroll
+    for (int t = 0; t < kAhead; ++t) {  // slots always exist; which of them were written is decided below
+        ml[t] = *reinterpret_cast<const float2 *>(slot[t] + 16 * D + 2 * r);
+        const float *ps = slot[t] + r * D + lane * PER;
+        if constexpr (PER == 2) {
+            const float2 x = *reinterpret_cast<const float2 *>(ps);
+            v[t][0] = x.x;
+            v[t][1] = x.y;
+        } else {
+            const float4 x = *reinterpret_cast<const float4 *>(ps);
+            v[t][0] = x.x;
+            v[t][1] = x.y;
+            v[t][PER - 2] = x.z;
+            v[t][PER - 1] = x.w;
+        }
+    }
+    const int ntiles = (max(0, min(pl_raw, P.pl_max)) + P.K + TK - 1) / TK;
+
     float acc[PER];
 #pragma unroll
     for (int c = 0; c < PER; ++c) acc[c] = 0.f;
     float mm = -CUDART_INF_F, ll = 0.f;
-    for (int gg = g_first; gg <= g_last; ++gg) {
-        const long long sb = share_begin(gg, T, P.workers);
-        const long long seg_begin = sb > a ? sb : a;
-        if (seg_begin - a >= ntiles) break;  // this share and all later ones saw no visible key of the item
-        const int slot = a <= sb ? 0 : 1;
-        const float *slot_base = P.part + (static_cast<size_t>(gg) * 2 + slot) * 16 * (D + 2);
-        const float *ps = slot_base + r * D + lane * PER;  // 16-byte aligned for D = 128, 8-byte for D = 64
-        const float2 ml = *reinterpret_cast<const float2 *>(slot_base + 16 * D + 2 * r);
-        float v[PER];
-        if constexpr (PER == 2) {
-            const float2 t = *reinterpret_cast<const float2 *>(ps);
-            v[0] = t.x;
-            v[1] = t.y;
-        } else {
-            const float4 t = *reinterpret_cast<const float4 *>(ps);
-            v[0] = t.x;
-            v[1] = t.y;
-            v[PER - 2] = t.z;
-            v[PER - 1] = t.w;
-        }
-        const float mn = fmaxf(mm, ml.x);
+    auto fold = [&](float2 m_l, const float (&val)[PER]) {
+        const float mn = fmaxf(mm, m_l.x);
         const float mu = mn == -CUDART_INF_F ? 0.f : mn;
-        const float f_old = fast_exp2(mm - mu), f_new = fast_exp2(ml.x - mu);
+        const float f_old = fast_exp2(mm - mu), f_new = fast_exp2(m_l.x - mu);
         mm = mn;
-        ll = ll * f_old + ml.y * f_new;
+        ll = ll * f_old + m_l.y * f_new;
 #pragma unroll
-        for (int c = 0; c < PER; ++c) acc[c] = acc[c] * f_old + v[c] * f_new;
+        for (int c = 0; c < PER; ++c) acc[c] = acc[c] * f_old + val[c] * f_new;
+    };
+    // a share whose part of the item starts past the stream's last visible key wrote nothing
+#pragma unroll
+    for (int t = 0; t < kAhead; ++t)
+        if (g_first + t <= g_last && seg_off[t] < ntiles) fold(ml[t], v[t]);
+    for (int gg = g_first + kAhead; gg <= g_last; ++gg) {  // items spread over more shares than that: one by one
+        const long long sb = share_begin(gg, T, P.workers);
+        if ((sb > a ? sb : a) - a >= ntiles) break;
+        const float *sl = P.part + (static_cast<size_t>(gg) * 2 + (a <= sb ? 0 : 1)) * 16 * (D + 2);
+        const float2 m_l = *reinterpret_cast<const float2 *>(sl + 16 * D + 2 * r);
+        float val[PER];
+#pragma unroll
+        for (int c = 0; c < PER; ++c) val[c] = sl[r * D + lane * PER + c];
+        fold(m_l, val);
     }
     const float inv = 1.f / ll;
     const int h = hk * group + chunk * P.chunk_heads + r / P.K, i = r % P.K;
