@@ -43,6 +43,7 @@ def _load():
             _lib.hawk_oracle_cfg_accept.restype = ctypes.c_int
             _lib.hawk_oracle_target_probs.restype = ctypes.c_int
             _lib.hawk_oracle_target_probs_rows.restype = ctypes.c_int
+            _lib.hawk_oracle_tree_accept.restype = ctypes.c_int
     return _lib
 
 
@@ -136,4 +137,30 @@ def cfg_accept(logits, q_probs, draft, u_accept, u_resample, v_begin, v_end, cfg
         ctypes.c_float(cfg_scale), ctypes.c_float(temperature), int(top_k), int(bool(has_bonus_row)),
         _p(accept_len), _p(token), _p(ratio), _p(acc_margin), _p(res_margin))
     return dict(accept_len=accept_len, token=token, ratio=ratio, accept_margin=acc_margin,
+                resample_margin=res_margin, flags=flags)
+
+
+def tree_accept(logits, q_probs, node_token, node_q, child_begin, u_accept, u_resample, v_begin, v_end,
+                cfg_scale, temperature, top_k, max_depth=None, diagnostics=True) -> dict:
+    """Verification of a candidate tree; see hawk_oracle_tree_accept in the C source for the contract."""
+    logits = _c(logits, np.float32); q_probs = _c(q_probs, np.float32)
+    node_token = _c(node_token, np.int32); node_q = _c(node_q, np.int32)
+    child_begin = _c(child_begin, np.int32)
+    u_accept = _c(u_accept, np.float32); u_resample = _c(u_resample, np.float32)
+    B, NQ, V = q_probs.shape
+    N = node_q.shape[0]
+    assert logits.shape == (2 * B, N, V), (logits.shape, (2 * B, N, V))
+    assert node_token.shape == (B, N) and child_begin.shape == (N + 1,)
+    assert u_accept.shape == (B, N) and u_resample.shape == (B, N)
+    max_depth = N if max_depth is None else max_depth
+    accept_len = np.empty(B, dtype=np.int32)
+    token = np.empty(B, dtype=np.int32)
+    path = np.empty((B, max_depth), dtype=np.int32)
+    acc_margin = np.empty((B, N), dtype=np.float64) if diagnostics else None
+    res_margin = np.empty(B, dtype=np.float64) if diagnostics else None
+    flags = _load().hawk_oracle_tree_accept(
+        _p(logits), _p(q_probs), _p(node_token), _p(node_q), _p(child_begin), _p(u_accept), _p(u_resample),
+        B, N, NQ, V, v_begin, v_end, ctypes.c_float(cfg_scale), ctypes.c_float(temperature), int(top_k),
+        _p(accept_len), _p(token), _p(path), max_depth, _p(acc_margin), _p(res_margin))
+    return dict(accept_len=accept_len, token=token, path=path, accept_margin=acc_margin,
                 resample_margin=res_margin, flags=flags)

@@ -16,7 +16,10 @@
  * Parity pins (tests marked "not gpu"): brute-force attention, uniform-weights closed form,
  * causality, numpy GEMM, identity weight, softmax special cases, q == p accepts all, disjoint
  * support accepts none, acceptance rate = sum min(p,q), distribution-preservation identity,
- * chi-square of the emitted token, inverse-CDF end points, a hand-computed worked example.
+ * chi-square of the emitted token, inverse-CDF end points, a hand-computed worked example; for the
+ * candidate tree: a hand-computed walk, equality with the chain on chain-shaped trees, chi-square of
+ * the first emitted token with three different draft heads, all-rejected rate = prod(1 - alpha_j),
+ * candidates drawn from the (refined) target always pass.
  * Nothing here is "parity unpinned".
  *
  * OpenMP is used only across independent units (stream x head, token row, sequence).
@@ -325,5 +328,96 @@ int hawk_oracle_target_probs_rows(const float *logits, int B, int rows, int V, i
             all_flags |= hawk_oracle_target_probs(lc, lu, V, v_begin, v_end, cfg_scale, temperature,
                                                   top_k, p_out + ((size_t)b * rows + i) * (size_t)V);
         }
+    return all_flags;
+}
+
+/* ------------------------------------------------------------------------------------------
+ * Step 3 with several candidates per depth: verification of a candidate TREE (Sec. 4.2,
+ * "Sampling and Verification", Eq. "recur"; proof of distribution preservation in App. A).
+ * Candidates at the same depth are verified one after the other.  A candidate x drawn from its
+ * draft distribution q passes with probability min(1, p(x)/q(x)); when it passes, decoding moves to
+ * that node and one level deeper; each rejection replaces the target by
+ *     p <- norm(max(0, p - q))            (q: the distribution the rejected candidate came from)
+ * and when every candidate of a level is rejected (or the node has none), the correction token is
+ * drawn from the target as refined so far.  q may differ from candidate to candidate (horizontal or
+ * vertical draft head).  A residual without mass (p <= q everywhere) leaves p as it is.
+ *
+ * The tree is shared by the batch.  Node 0 is the root (the last committed token); the children of
+ * node n are the nodes child_begin[n] .. child_begin[n+1]-1, in verification order.
+ *   logits      fp32 [2B][N][V]  row n: target logits for the token that follows node n
+ *   q_probs     fp32 [B][NQ][V]  draft distributions
+ *   node_token  int32 [B][N]     candidate token of node n (entry 0 unused)
+ *   node_q      int32 [N]        row of q_probs that node n's token was drawn from (entry 0 unused)
+ *   child_begin int32 [N+1]
+ *   u_accept    fp32 [B][N]      one uniform per candidate node (entry 0 unused)
+ *   u_resample  fp32 [B][N]      entry n drives the draw if the walk stops at node n
+ *   accept_len  int32 [B]        number of accepted candidates = depth of the node the walk stops at
+ *   out_token   int32 [B]        the correction token (-1 if the refined target has no mass at all)
+ *   path        int32 [B][max_depth]  accepted nodes in order, -1 beyond accept_len (may be NULL)
+ * Optional diagnostics (may be NULL): accept_margin fp64 [B][N] = |u - min(1, p(x)/q(x))| of every
+ * candidate examined (inf otherwise); resample_margin fp64 [B].
+ * returns OR of flags.
+ * ------------------------------------------------------------------------------------------ */
+int hawk_oracle_tree_accept(const float *logits, const float *q_probs, const int32_t *node_token,
+                            const int32_t *node_q, const int32_t *child_begin,
+                            const float *u_accept, const float *u_resample, int B, int N, int NQ,
+                            int V, int v_begin, int v_end, float cfg_scale, float temperature,
+                            int top_k, int32_t *accept_len, int32_t *out_token, int32_t *path,
+                            int max_depth, double *accept_margin, double *resample_margin)
+{
+    int all_flags = 0;
+    (void)NQ;
+#pragma omp parallel for schedule(dynamic) reduction(| : all_flags)
+    for (int b = 0; b < B; ++b) {
+        double *p = (double *)malloc(sizeof(double) * (size_t)V);
+        double *r = (double *)malloc(sizeof(double) * (size_t)V);
+        int flags = 0, n = 0, depth = 0;
+        if (resample_margin) resample_margin[b] = INFINITY;
+        if (accept_margin)
+            for (int c = 0; c < N; ++c) accept_margin[(size_t)b * N + c] = INFINITY;
+        if (path)
+            for (int d = 0; d < max_depth; ++d) path[(size_t)b * max_depth + d] = -1;
+        for (;;) {
+            const float *lc = logits + ((size_t)b * N + n) * (size_t)V;
+            const float *lu = logits + ((size_t)(B + b) * N + n) * (size_t)V;
+            flags |= hawk_oracle_target_probs(lc, lu, V, v_begin, v_end, cfg_scale, temperature,
+                                              top_k, p);
+            int next = -1;
+            for (int c = child_begin[n]; c < child_begin[n + 1] && next < 0; ++c) {
+                const float *q = q_probs + ((size_t)b * NQ + node_q[c]) * (size_t)V;
+                int x = node_token[(size_t)b * N + c];
+                if (x < v_begin || x >= v_end) {
+                    flags |= ORACLE_FLAG_BAD_DRAFT;
+                    x = x < v_begin ? v_begin : v_end - 1;
+                }
+                double u = (double)u_accept[(size_t)b * N + c];
+                double qx = (double)q[x], px = p[x];
+                if (accept_margin) {
+                    double rr = qx > 0.0 ? px / qx : (px > 0.0 ? INFINITY : 0.0);
+                    accept_margin[(size_t)b * N + c] = fabs(u - (rr < 1.0 ? rr : 1.0));
+                }
+                if (u * qx < px) {
+                    next = c;                                  /* passed: one level deeper */
+                    break;
+                }
+                double total = hawk_oracle_residual(p, q, V, v_begin, v_end, r);
+                if (total > 0.0)                               /* p <- norm(max(0, p - q)) */
+                    for (int v = v_begin; v < v_end; ++v) p[v] = r[v] / total;
+            }
+            if (next >= 0) {
+                if (path && depth < max_depth) path[(size_t)b * max_depth + depth] = next;
+                ++depth;
+                n = next;
+                continue;
+            }
+            accept_len[b] = depth;
+            out_token[b] = inverse_cdf(p, v_begin, v_end, (double)u_resample[(size_t)b * N + n], 1.0,
+                                       resample_margin ? &resample_margin[b] : NULL);
+            break;
+        }
+        all_flags |= flags;
+        free(p);
+        free(r);
+    }
     return all_flags;
 }
