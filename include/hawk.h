@@ -8,7 +8,8 @@
  *                     the conditional and the unconditional guidance stream;
  *   hawk_head_proj    projection of the K hidden states onto the image-token codebook;
  *   hawk_cfg_accept   guidance combine, temperature, top-k, softmax and speculative rejection
- *                     sampling, returning the accepted length and the correction token.
+ *                     sampling, returning the accepted length and the correction token;
+ *   hawk_tree_accept  the same for a candidate tree with several candidates per depth.
  *
  * Conventions common to all entry points
  *   - Every pointer is a DEVICE pointer owned by the caller unless the comment says "host".  The
@@ -51,6 +52,7 @@ typedef enum {
 #define HAWK_DEV_BAD_DRAFT 2  /* a draft id lay outside [v_begin, v_end) and was clamped into it */
 #define HAWK_DEV_NONFINITE 4  /* a NaN or +inf logit was treated as -inf                        */
 #define HAWK_DEV_BAD_PREFIX 8 /* a prefix length lay outside [0, L_cap - K] and was clamped     */
+#define HAWK_DEV_BAD_TREE 16  /* a child range or draft-row index of the tree was out of range    */
 
 const char *hawk_status_string(hawk_status status);
 int hawk_version(void); /* major*10000 + minor*100 + patch */
@@ -151,6 +153,49 @@ hawk_status hawk_cfg_accept(const float *logits, const float *q_probs, const int
                             int has_bonus_row, int32_t *accept_len, int32_t *out_token,
                             float *p_debug, void *workspace, size_t workspace_bytes,
                             int32_t *dev_status, hawk_stream_t stream);
+
+/* ------------------------------------------------------------------------------------------------
+ * hawk_tree_accept - verification of a candidate tree: several candidates per depth, each with its
+ * own draft distribution.
+ *
+ * Operation (Sec. 4.2, "Sampling and Verification", Eq. "recur"; distribution preservation: App. A).
+ * The tree is shared by the batch: node 0 is the root (the last committed token), the children of
+ * node n are the nodes child_begin[n] .. child_begin[n+1]-1 (all ids > n), verified in that order.
+ * Per sequence b, starting at the root with depth 0:
+ *   1. p = target distribution of the node's logit rows (steps 1-3 of hawk_cfg_accept).
+ *   2. For each child c in order, with x = node_token[b][c], q = q_probs[b][node_q[c]]:
+ *      accept iff u_accept[b][c] * q[x] < p[x]; on a pass move to node c, one level deeper, step 1.
+ *      On a rejection p <- norm(max(0, p - q)); a residual without mass leaves p as it is.
+ *   3. Every child rejected, or the node has none: out_token[b] = inverse-CDF draw (ascending id)
+ *      from p as refined so far with u_resample[b][node]; accept_len[b] = depth; stop.
+ * q may come from a different draft head for every candidate (horizontal or vertical), which is what
+ * shrinks the probability that all candidates of a level are rejected.
+ * A chain of K drafts is the tree with N = K + 1 nodes and child_begin[n] = n + 1.
+ *
+ *   logits      fp32 [2B][N][V]  row n: logits for the token that follows node n (b conditional, B+b not)
+ *   q_probs     fp32 [B][NQ][V]  draft probabilities, used as given
+ *   node_token  int32 [B][N]     candidate token of node n (entry 0 unused)
+ *   node_q      int32 [N]        row of q_probs the token of node n was drawn from (entry 0 unused)
+ *   child_begin int32 [N+1]      device memory, like everything else
+ *   u_accept    fp32 [B][N]      uniforms in [0,1), one per candidate node (entry 0 unused)
+ *   u_resample  fp32 [B][N]      uniforms in [0,1), entry n used if the walk stops at node n
+ *   accept_len  int32 [B] (out)  number of accepted candidates
+ *   out_token   int32 [B] (out)  correction token; -1 if the refined target has no mass at all
+ *   path        optional int32 [B][max_depth] (out): accepted nodes in order, -1 beyond accept_len
+ *   workspace   at least hawk_tree_accept_workspace_bytes(B, N) bytes, 16-byte aligned, no initialisation
+ * Every node is judged by its own thread block whether or not the walk reaches it, so the cost is
+ * B*N rows.  Supported: 1 <= N <= 65536; at most 16 children per node; valid ids as hawk_cfg_accept.
+ * A child range that breaks these rules is clamped and flagged HAWK_DEV_BAD_TREE; the walk always ends.
+ * Errors: NULL, SHAPE, ALIGN, UNSUPPORTED, WORKSPACE, PARAM, CUDA.  B == 0 returns HAWK_OK.
+ * ---------------------------------------------------------------------------------------------- */
+size_t hawk_tree_accept_workspace_bytes(int B, int N);
+
+hawk_status hawk_tree_accept(const float *logits, const float *q_probs, const int32_t *node_token,
+                             const int32_t *node_q, const int32_t *child_begin, const float *u_accept,
+                             const float *u_resample, int B, int N, int NQ, int V, int v_begin, int v_end,
+                             float cfg_scale, float temperature, int top_k, int max_depth,
+                             int32_t *accept_len, int32_t *out_token, int32_t *path, void *workspace,
+                             size_t workspace_bytes, int32_t *dev_status, hawk_stream_t stream);
 
 /* ------------------------------------------------------------------------------------------------
  * hawk_cfg_accept_noalloc - hawk_cfg_accept without a caller-provided workspace.

@@ -12,7 +12,7 @@ _BINDING_NAMES = (
     "verify_attn", "verify_attn_workspace_bytes", "head_proj",
     "cfg_accept", "cfg_accept_workspace_bytes",
     "verify_step_host", "StepHostArgs",
-    "cfg_accept_noalloc", "cfg_accept_noalloc_max_rows",
+    "cfg_accept_noalloc", "cfg_accept_noalloc_max_rows", "tree_accept",
 )
 
 

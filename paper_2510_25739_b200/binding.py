@@ -16,7 +16,7 @@ _PKG = Path(__file__).resolve().parent
 _LIB_PATH = _PKG / "libhawk_verify.so"
 _lib: Optional[ctypes.CDLL] = None
 
-DEV_TIMEOUT, DEV_BAD_DRAFT, DEV_NONFINITE, DEV_BAD_PREFIX = 1, 2, 4, 8
+DEV_TIMEOUT, DEV_BAD_DRAFT, DEV_NONFINITE, DEV_BAD_PREFIX, DEV_BAD_TREE = 1, 2, 4, 8, 16
 
 EXPORTS = (
     "hawk_status_string", "hawk_version",
@@ -25,6 +25,7 @@ EXPORTS = (
     "hawk_cfg_accept_workspace_bytes", "hawk_cfg_accept",
     "hawk_verify_step_host",
     "hawk_cfg_accept_noalloc_max_rows", "hawk_cfg_accept_noalloc",
+    "hawk_tree_accept_workspace_bytes", "hawk_tree_accept",
 )
 
 
@@ -87,6 +88,10 @@ def load_library() -> ctypes.CDLL:
     lib.hawk_cfg_accept_noalloc.restype = i32
     lib.hawk_cfg_accept_noalloc.argtypes = [vp, vp, vp, vp, vp, i32, i32, i32, i32, i32, f32, f32, i32, i32,
                                             vp, vp, vp, vp]
+    lib.hawk_tree_accept_workspace_bytes.restype = sz
+    lib.hawk_tree_accept_workspace_bytes.argtypes = [i32, i32]
+    lib.hawk_tree_accept.restype = i32
+    lib.hawk_tree_accept.argtypes = [vp] * 7 + [i32] * 6 + [f32, f32, i32, i32] + [vp, vp, vp, vp, sz, vp, vp]
     lib.hawk_verify_step_host.restype = i32
     lib.hawk_verify_step_host.argtypes = [ctypes.POINTER(StepHostArgs), vp]
     _lib = lib
@@ -237,6 +242,39 @@ def cfg_accept_noalloc(logits: torch.Tensor, q_probs: torch.Tensor, draft: torch
     if rc != 0:
         raise HawkError(rc, "hawk_cfg_accept_noalloc")
     return accept_len, out_token
+
+
+def tree_accept(logits: torch.Tensor, q_probs: torch.Tensor, node_token: torch.Tensor, node_q: torch.Tensor,
+                child_begin: torch.Tensor, u_accept: torch.Tensor, u_resample: torch.Tensor, v_begin: int,
+                v_end: int, cfg_scale: float, temperature: float, top_k: int, max_depth: Optional[int] = None,
+                dev_status: Optional[torch.Tensor] = None):
+    """Candidate-tree verification: logits [2B,N,V], q_probs [B,NQ,V], node_token [B,N], node_q [N],
+    child_begin [N+1], uniforms [B,N] -> (accept_len [B], out_token [B], path [B,max_depth])."""
+    lib = load_library()
+    B, NQ, V = q_probs.shape
+    N = node_q.shape[0]
+    max_depth = N if max_depth is None else int(max_depth)
+    _check(logits, torch.float32, "logits", (2 * B, N, V))
+    _check(q_probs, torch.float32, "q_probs")
+    _check(node_token, torch.int32, "node_token", (B, N))
+    _check(node_q, torch.int32, "node_q", (N,))
+    _check(child_begin, torch.int32, "child_begin", (N + 1,))
+    _check(u_accept, torch.float32, "u_accept", (B, N))
+    _check(u_resample, torch.float32, "u_resample", (B, N))
+    dev = logits.device
+    accept_len = torch.empty(B, dtype=torch.int32, device=dev)
+    out_token = torch.empty(B, dtype=torch.int32, device=dev)
+    path = torch.empty((B, max_depth), dtype=torch.int32, device=dev)
+    need = int(lib.hawk_tree_accept_workspace_bytes(B, N))
+    workspace = torch.empty(max(need, 16), dtype=torch.uint8, device=dev)
+    rc = lib.hawk_tree_accept(_ptr(logits), _ptr(q_probs), _ptr(node_token), _ptr(node_q), _ptr(child_begin),
+                              _ptr(u_accept), _ptr(u_resample), B, N, NQ, V, int(v_begin), int(v_end),
+                              float(cfg_scale), float(temperature), int(top_k), max_depth, _ptr(accept_len),
+                              _ptr(out_token), _ptr(path), _ptr(workspace), workspace.numel(), _ptr(dev_status),
+                              _stream())
+    if rc != 0:
+        raise HawkError(rc, "hawk_tree_accept")
+    return accept_len, out_token, path
 
 
 def verify_step_host(args: StepHostArgs) -> None:

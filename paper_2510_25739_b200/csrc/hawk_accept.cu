@@ -158,42 +158,35 @@ __device__ __forceinline__ T block_exclusive_scan(T v, T *scratch32, T *total)
     return __shfl_sync(0xffffffffu, wi - w, warp) + (incl - v);
 }
 
-// NT threads, VPT float4 loads per thread: the block holds up to 4 * NT * VPT valid ids of its row.
+constexpr int kMaxChildren = 16;  // candidates verified at one tree node, at most
+
+// Shared memory of one row block.
 template <int NT, int VPT>
-__global__ void __launch_bounds__(NT) accept_rows_kernel(const AcceptParams P)
+struct RowShared {
+    int hist[kBins];
+    float cand[kCandMax];
+    Scratch<NT> red;
+    float wt[VPT * (NT / 32)];
+    float wbase[VPT * (NT / 32)];
+    int bin, above, tok;
+    float tau, pxe, total;
+    int ctok[kMaxChildren];
+    float cqx[kMaxChildren], cu[kMaxChildren];
+};
+
+// Reads the conditional and unconditional logit rows once and leaves the guided logits of the block's
+// ids in registers (id of x[j][c]: 4 * (j * NT + tid) + c; ids past n hold -inf); also this thread's
+// max, min and count of finite values.
+template <int NT, int VPT>
+__device__ __forceinline__ void row_load(const float *lc, const float *lu, int n, bool vec_ok, float cfg_scale,
+                                         float temperature, float (&x)[VPT][4], float &mx, float &mn, int &cnt,
+                                         int &flags)
 {
     constexpr int NW = NT / 32;
-    constexpr int BPT = kBins / NT;  // histogram bins per thread
-    static_assert(kBins % NT == 0 && BPT >= 1, "bins must split evenly over the block");
-    static_assert(VPT * NW <= NT, "warp totals of the scan must fit one block-wide scan");
-
-    __shared__ int s_hist[kBins];
-    __shared__ float s_cand[kCandMax];
-    __shared__ Scratch<NT> s_red;
-    __shared__ float s_wt[VPT * NW];
-    __shared__ float s_wbase[VPT * NW];
-    __shared__ int s_bin, s_above, s_tok;
-    __shared__ float s_tau, s_pxe, s_total;
-
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    hawk::allow_dependent_launch();
-    hawk::grid_dependency_wait();
-
-    const int row = blockIdx.x;  // position-major: all rows of position 0 first
-    const int i = row / P.B, b = row - i * P.B;
-    const bool bonus = (i == P.K);
-    const int n = P.n;
-    const bool vec_ok = P.vec_ok != 0;
-    const float *lc = P.logits + (static_cast<size_t>(b) * P.rows + i) * P.V + P.v_begin;
-    const float *lu = P.logits + (static_cast<size_t>(P.B + b) * P.rows + i) * P.V + P.v_begin;
-    const float *qrow = bonus ? nullptr : P.q + (static_cast<size_t>(b) * P.K + i) * P.V + P.v_begin;
-    int flags = 0;
-
-    const bool unit_T = P.temperature == 1.0f;
-    // ---- read both logit rows once, combine into registers
-    float x[VPT][4];
-    float mx = -CUDART_INF_F, mn = CUDART_INF_F;
-    int cnt = 0;
+    (void)lane; (void)warp; (void)NW;
+    const bool unit_T = temperature == 1.0f;
+    mx = -CUDART_INF_F, mn = CUDART_INF_F, cnt = 0;
     {
         float4 c4[VPT], u4[VPT];
 #pragma unroll
@@ -206,10 +199,10 @@ __global__ void __launch_bounds__(NT) accept_rows_kernel(const AcceptParams P)
         for (int j = 0; j < VPT; ++j) {
             const int e0 = 4 * (j * NT + tid);
             int fl = 0;
-            x[j][0] = e0 + 0 < n ? guided(c4[j].x, u4[j].x, P.cfg_scale, P.temperature, unit_T, fl) : -CUDART_INF_F;
-            x[j][1] = e0 + 1 < n ? guided(c4[j].y, u4[j].y, P.cfg_scale, P.temperature, unit_T, fl) : -CUDART_INF_F;
-            x[j][2] = e0 + 2 < n ? guided(c4[j].z, u4[j].z, P.cfg_scale, P.temperature, unit_T, fl) : -CUDART_INF_F;
-            x[j][3] = e0 + 3 < n ? guided(c4[j].w, u4[j].w, P.cfg_scale, P.temperature, unit_T, fl) : -CUDART_INF_F;
+            x[j][0] = e0 + 0 < n ? guided(c4[j].x, u4[j].x, cfg_scale, temperature, unit_T, fl) : -CUDART_INF_F;
+            x[j][1] = e0 + 1 < n ? guided(c4[j].y, u4[j].y, cfg_scale, temperature, unit_T, fl) : -CUDART_INF_F;
+            x[j][2] = e0 + 2 < n ? guided(c4[j].z, u4[j].z, cfg_scale, temperature, unit_T, fl) : -CUDART_INF_F;
+            x[j][3] = e0 + 3 < n ? guided(c4[j].w, u4[j].w, cfg_scale, temperature, unit_T, fl) : -CUDART_INF_F;
             flags |= fl;
 #pragma unroll
             for (int c = 0; c < 4; ++c)
@@ -220,38 +213,23 @@ __global__ void __launch_bounds__(NT) accept_rows_kernel(const AcceptParams P)
                 }
         }
     }
-    // draft id, its q and the uniforms
-    int xd = 0;
-    float qx = 0.f, u_acc = 0.f;
-    if (!bonus) {
-        xd = P.draft[b * P.K + i];
-        if (xd < P.v_begin || xd >= P.v_begin + n) {
-            flags |= HAWK_DEV_BAD_DRAFT;
-            xd = xd < P.v_begin ? P.v_begin : P.v_begin + n - 1;
-        }
-        xd -= P.v_begin;
-        qx = qrow[xd];
-        u_acc = P.u_acc[b * P.K + i];
-    }
-    const float u_res = P.u_res[b * (P.K + 1) + i];
-    if (flags && P.dev_status) atomicOr(P.dev_status, flags);
+}
 
-    block_minmaxcount<NT>(mx, mn, cnt, s_red);
-
-    if (cnt == 0) {  // nothing has mass: p == 0 everywhere, the draft is rejected, no token exists
-        if (P.p_debug) {
-            float *pd = P.p_debug + (static_cast<size_t>(b) * P.rows + i) * P.V + P.v_begin;
-            for (int e = tid; e < n; e += NT) pd[e] = 0.f;
-        }
-        if (tid == 0) P.row_out[b * P.rows + i] = ROW_REJECTED_NO_TOKEN;
-        return;
-    }
-
-    // ---- top-k threshold: the top_k-th largest finite value (exact; ties at it are all kept)
+// Top-k threshold of a row held in registers: the top_k-th largest finite value (exact; ties at it
+// are all kept).  -inf when nothing is to be filtered.  mn, mx, cnt: block-wide range and count.
+template <int NT, int VPT>
+__device__ __forceinline__ float row_topk(const float (&x)[VPT][4], float mn, float mx, int cnt, int top_k,
+                                          RowShared<NT, VPT> &sh)
+{
+    constexpr int BPT = kBins / NT;  // histogram bins per thread
+    static_assert(kBins % NT == 0 && BPT >= 1, "bins must split evenly over the block");
+    constexpr int NW = NT / 32;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    (void)lane; (void)warp; (void)NW;
     float tau = -CUDART_INF_F;
-    if (P.top_k > 0 && P.top_k < cnt) {
+    if (top_k > 0 && top_k < cnt) {
         float lo = mn, hi = mx;
-        int k = P.top_k;
+        int k = top_k;
         for (int round = 0; round < kMaxRounds; ++round) {
             if (!(hi > lo)) {
                 tau = hi;
@@ -260,7 +238,7 @@ __global__ void __launch_bounds__(NT) accept_rows_kernel(const AcceptParams P)
             // histogram of the values in [lo, hi]: bin 0 holds the largest
             const float scale = static_cast<float>(kBins) / (hi - lo);
 #pragma unroll
-            for (int t = 0; t < BPT; ++t) s_hist[t * NT + tid] = 0;
+            for (int t = 0; t < BPT; ++t) sh.hist[t * NT + tid] = 0;
             __syncthreads();
             int bins[VPT][4];  // bin of every value held (-1: outside [lo, hi])
 #pragma unroll
@@ -270,28 +248,28 @@ __global__ void __launch_bounds__(NT) accept_rows_kernel(const AcceptParams P)
                     const float v = x[j][c];
                     const bool in = v >= lo && v <= hi;
                     bins[j][c] = in ? min(kBins - 1, static_cast<int>((hi - v) * scale)) : -1;
-                    if (in) atomicAdd(&s_hist[bins[j][c]], 1);
+                    if (in) atomicAdd(&sh.hist[bins[j][c]], 1);
                 }
             __syncthreads();
             int local = 0;
 #pragma unroll
-            for (int t = 0; t < BPT; ++t) local += s_hist[tid * BPT + t];
+            for (int t = 0; t < BPT; ++t) local += sh.hist[tid * BPT + t];
             int total;
-            const int excl = block_exclusive_scan<NT, int>(local, s_red.iscan, &total);
+            const int excl = block_exclusive_scan<NT, int>(local, sh.red.iscan, &total);
             if (excl < k && k <= excl + local) {  // exactly one thread: one of its bins holds the k-th largest
                 int run = excl;
 #pragma unroll
                 for (int t = 0; t < BPT; ++t) {
-                    const int h = s_hist[tid * BPT + t];
+                    const int h = sh.hist[tid * BPT + t];
                     if (run < k && k <= run + h) {
-                        s_bin = tid * BPT + t;
-                        s_above = run;
+                        sh.bin = tid * BPT + t;
+                        sh.above = run;
                     }
                     run += h;
                 }
             }
             __syncthreads();
-            const int bstar = s_bin, kk = k - s_above, C = s_hist[bstar];
+            const int bstar = sh.bin, kk = k - sh.above, C = sh.hist[bstar];
             if (C <= kCandMax) {
                 // rank the members of the bin exactly: the kk-th largest of them is the threshold.
                 // They are compacted into shared memory by a prefix sum over the threads' member counts
@@ -302,40 +280,40 @@ __global__ void __launch_bounds__(NT) accept_rows_kernel(const AcceptParams P)
 #pragma unroll
                     for (int c = 0; c < 4; ++c) mine += bins[j][c] == bstar;
                 int ctotal;
-                int pos = block_exclusive_scan<NT, int>(mine, s_red.iscan, &ctotal);
+                int pos = block_exclusive_scan<NT, int>(mine, sh.red.iscan, &ctotal);
                 if (mine) {
 #pragma unroll
                     for (int j = 0; j < VPT; ++j)
 #pragma unroll
                         for (int c = 0; c < 4; ++c)
-                            if (bins[j][c] == bstar) s_cand[pos++] = x[j][c];
+                            if (bins[j][c] == bstar) sh.cand[pos++] = x[j][c];
                 }
                 __syncthreads();
                 if (C <= 32) {  // the usual case: one warp ranks them with shuffles
                     if (warp == 0) {
-                        const float v = lane < C ? s_cand[lane] : -CUDART_INF_F;
+                        const float v = lane < C ? sh.cand[lane] : -CUDART_INF_F;
                         int gt = 0, ge = 0;
                         for (int m = 0; m < C; ++m) {
                             const float w = __shfl_sync(0xffffffffu, v, m);
                             gt += w > v;
                             ge += w >= v;
                         }
-                        if (lane < C && gt < kk && kk <= ge) s_tau = v;
+                        if (lane < C && gt < kk && kk <= ge) sh.tau = v;
                     }
                 } else {
                     for (int t = tid; t < C; t += NT) {
-                        const float v = s_cand[t];
+                        const float v = sh.cand[t];
                         int gt = 0, ge = 0;
                         for (int m = 0; m < C; ++m) {
-                            const float w = s_cand[m];
+                            const float w = sh.cand[m];
                             gt += w > v;
                             ge += w >= v;
                         }
-                        if (gt < kk && kk <= ge) s_tau = v;  // several threads may hold the same value
+                        if (gt < kk && kk <= ge) sh.tau = v;  // several threads may hold the same value
                     }
                 }
                 __syncthreads();
-                tau = s_tau;
+                tau = sh.tau;
                 break;
             }
             // too many members share the bin: narrow the range to their values and repeat
@@ -349,7 +327,7 @@ __global__ void __launch_bounds__(NT) accept_rows_kernel(const AcceptParams P)
                         nmx = fmaxf(nmx, x[j][c]);
                         nmn = fminf(nmn, x[j][c]);
                     }
-            block_minmaxcount<NT>(nmx, nmn, dummy, s_red);
+            block_minmaxcount<NT>(nmx, nmn, dummy, sh.red);
             lo = nmn;
             hi = nmx;
             k = kk;
@@ -357,7 +335,13 @@ __global__ void __launch_bounds__(NT) accept_rows_kernel(const AcceptParams P)
         }
     }
 
-    // ---- softmax over what is kept: x becomes exp(l - max), unnormalised
+    return tau;
+}
+
+// x becomes exp(l - max) for the ids kept by the threshold (0 for the others); returns the block-wide sum.
+template <int NT, int VPT>
+__device__ __forceinline__ float row_softmax(float (&x)[VPT][4], float tau, float mx, RowShared<NT, VPT> &sh)
+{
     constexpr float kLog2e = 1.4426950408889634f;
     float zsum = 0.f;
 #pragma unroll
@@ -369,15 +353,181 @@ __global__ void __launch_bounds__(NT) accept_rows_kernel(const AcceptParams P)
             x[j][c] = e;
             zsum += e;
         }
-    if (!bonus && tid == ((xd >> 2) % NT)) {  // the thread that holds the draft id
+    return block_sum<NT>(zsum, sh.red);
+}
+
+// Running sums of the non-negative weights rr in ascending id order: sj = sum of each group of 4,
+// incl = inclusive scan of sj over the warp, sh.wbase = mass before each (group row, warp); returns the
+// total mass.  Also resets sh.tok for row_search().
+template <int NT, int VPT>
+__device__ __forceinline__ float row_mass(const float (&rr)[VPT][4], float (&sj)[VPT], float (&incl)[VPT],
+                                          RowShared<NT, VPT> &sh)
+{
+    static_assert(VPT * (NT / 32) <= NT, "warp totals of the scan must fit one block-wide scan");
+    constexpr int NW = NT / 32;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    (void)lane; (void)warp; (void)NW;
+#pragma unroll
+    for (int j = 0; j < VPT; ++j) sj[j] = ((rr[j][0] + rr[j][1]) + rr[j][2]) + rr[j][3];
+#pragma unroll
+    for (int j = 0; j < VPT; ++j) {
+        float v = sj[j];
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const float up = __shfl_up_sync(0xffffffffu, v, o);
+            if (lane >= o) v += up;
+        }
+        incl[j] = v;
+        if (lane == 31) sh.wt[j * NW + warp] = v;
+    }
+    __syncthreads();
+    if (warp == 0) {  // exclusive prefix of the VPT * NW warp totals (ascending id order), by one warp
+        constexpr int E = VPT * NW, PER = (E + 31) / 32;
+        float ent[PER], run = 0.f;
+#pragma unroll
+        for (int t = 0; t < PER; ++t) {
+            ent[t] = lane * PER + t < E ? sh.wt[lane * PER + t] : 0.f;
+            run += ent[t];
+        }
+        float incl_l = run;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const float up = __shfl_up_sync(0xffffffffu, incl_l, o);
+            if (lane >= o) incl_l += up;
+        }
+        float base = incl_l - run;
+#pragma unroll
+        for (int t = 0; t < PER; ++t) {
+            if (lane * PER + t < E) sh.wbase[lane * PER + t] = base;
+            base += ent[t];
+        }
+        if (lane == 31) sh.total = incl_l;
+        if (lane == 0) sh.tok = 0x7fffffff;
+    }
+    __syncthreads();
+    return sh.total;
+}
+
+// Inverse CDF: the smallest id (local to the valid range) whose running sum of rr exceeds tl; if
+// rounding leaves none, the last id with mass; -1 if no id has mass.
+template <int NT, int VPT>
+__device__ __forceinline__ int row_search(const float (&rr)[VPT][4], const float (&sj)[VPT],
+                                          const float (&incl)[VPT], float tl, RowShared<NT, VPT> &sh)
+{
+    constexpr int NW = NT / 32;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    (void)lane; (void)warp; (void)NW;
+    // pass 0: elements where the running sum crosses tl; pass 1 (only if the block-wide sums
+    // disagree at a thread boundary): the first element whose running sum exceeds tl
+    for (int pass = 0; pass < 2; ++pass) {
+#pragma unroll
+        for (int j = 0; j < VPT; ++j) {
+            const float excl = sh.wbase[j * NW + warp] + (incl[j] - sj[j]);
+            const bool look = pass == 0 ? (excl <= tl && excl + sj[j] > tl) : (excl + sj[j] > tl);
+            if (look) {
+                const int e0 = 4 * (j * NT + tid);
+                const float r0 = rr[j][0], r1 = rr[j][1], r2 = rr[j][2], r3 = rr[j][3];
+                const float c0 = excl + r0, c1 = excl + (r0 + r1), c2 = excl + ((r0 + r1) + r2);
+                const float c3 = excl + (((r0 + r1) + r2) + r3);
+                int hit = -1;  // an id without mass is never drawn
+                if (r0 > 0.f && c0 > tl) hit = 0;
+                else if (r1 > 0.f && c1 > tl) hit = 1;
+                else if (r2 > 0.f && c2 > tl) hit = 2;
+                else if (r3 > 0.f && c3 > tl) hit = 3;
+                if (hit >= 0) atomicMin(&sh.tok, e0 + hit);
+            }
+        }
+        __syncthreads();
+        if (sh.tok != 0x7fffffff) break;
+        __syncthreads();
+    }
+    int tok = sh.tok;
+    if (tok == 0x7fffffff) {  // rounding left no running sum above tl: the last id with mass
+        __syncthreads();
+        if (tid == 0) sh.tok = -1;
+        __syncthreads();
+#pragma unroll
+        for (int j = 0; j < VPT; ++j) {
+            const int e0 = 4 * (j * NT + tid);
+            if (sj[j] > 0.f) {
+                int last = -1;
+#pragma unroll
+                for (int c = 0; c < 4; ++c)
+                    if (rr[j][c] > 0.f) last = e0 + c;
+                if (last >= 0) atomicMax(&sh.tok, last);
+            }
+        }
+        __syncthreads();
+        tok = sh.tok;
+    }
+    return tok;
+}
+
+// Chain verification: one block per (sequence, draft position) row.
+// NT threads, VPT float4 loads per thread: the block holds up to 4 * NT * VPT valid ids of its row.
+template <int NT, int VPT>
+__global__ void __launch_bounds__(NT) accept_rows_kernel(const AcceptParams P)
+{
+    __shared__ RowShared<NT, VPT> sh;
+    const int tid = threadIdx.x;
+    hawk::allow_dependent_launch();
+    hawk::grid_dependency_wait();
+
+    const int row = blockIdx.x;  // position-major: all rows of position 0 first
+    const int i = row / P.B, b = row - i * P.B;
+    const bool bonus = (i == P.K);
+    const int n = P.n;
+    const bool vec_ok = P.vec_ok != 0;
+    const float *lc = P.logits + (static_cast<size_t>(b) * P.rows + i) * P.V + P.v_begin;
+    const float *lu = P.logits + (static_cast<size_t>(P.B + b) * P.rows + i) * P.V + P.v_begin;
+    const float *qrow = bonus ? nullptr : P.q + (static_cast<size_t>(b) * P.K + i) * P.V + P.v_begin;
+    int flags = 0;
+
+    // draft id and uniforms: requested before the rows, so that they have arrived when the rows have
+    int xd = bonus ? P.v_begin : P.draft[b * P.K + i];
+    const float u_acc = bonus ? 0.f : P.u_acc[b * P.K + i];
+    const float u_res = P.u_res[b * (P.K + 1) + i];
+
+    float x[VPT][4];
+    float mx, mn;
+    int cnt;
+    row_load<NT, VPT>(lc, lu, n, vec_ok, P.cfg_scale, P.temperature, x, mx, mn, cnt, flags);
+
+    float qx = 0.f;
+    if (!bonus) {
+        if (xd < P.v_begin || xd >= P.v_begin + n) {
+            flags |= HAWK_DEV_BAD_DRAFT;
+            xd = xd < P.v_begin ? P.v_begin : P.v_begin + n - 1;
+        }
+        xd -= P.v_begin;
+        qx = qrow[xd];
+    }
+    if (flags && P.dev_status) atomicOr(P.dev_status, flags);
+
+    block_minmaxcount<NT>(mx, mn, cnt, sh.red);
+
+    if (cnt == 0) {  // nothing has mass: p == 0 everywhere, the draft is rejected, no token exists
+        if (P.p_debug) {
+            float *pd = P.p_debug + (static_cast<size_t>(b) * P.rows + i) * P.V + P.v_begin;
+            for (int e = tid; e < n; e += NT) pd[e] = 0.f;
+        }
+        if (tid == 0) P.row_out[b * P.rows + i] = ROW_REJECTED_NO_TOKEN;
+        return;
+    }
+
+    const float tau = row_topk<NT, VPT>(x, mn, mx, cnt, P.top_k, sh);
+
+    // ---- softmax over what is kept: x becomes exp(l - max), unnormalised
+    if (!bonus && tid == ((xd >> 2) % NT)) {  // the thread that holds the draft id publishes exp(l_x - max)
 #pragma unroll
         for (int j = 0; j < VPT; ++j)
 #pragma unroll
             for (int c = 0; c < 4; ++c)
-                if (4 * (j * NT + tid) + c == xd) s_pxe = x[j][c];
+                if (4 * (j * NT + tid) + c == xd)
+                    sh.pxe = x[j][c] >= tau ? hawk::fast_exp2((x[j][c] - mx) * 1.4426950408889634f) : 0.f;
     }
-    const float Z = block_sum<NT>(zsum, s_red);
-    const float pxe = s_pxe;
+    const float Z = row_softmax<NT, VPT>(x, tau, mx, sh);  // its barriers publish sh.pxe
+    const float pxe = sh.pxe;
     const float invZ = 1.0f / Z;
 
     if (P.p_debug) {
@@ -391,7 +541,7 @@ __global__ void __launch_bounds__(NT) accept_rows_kernel(const AcceptParams P)
             }
     }
 
-    // ---- acceptance test on the draft token 
+    // ---- acceptance test on the draft token
     if (!bonus) {
         const float px = pxe * invZ;
         const bool accepted = static_cast<double>(u_acc) * static_cast<double>(qx) < static_cast<double>(px);
@@ -404,7 +554,7 @@ __global__ void __launch_bounds__(NT) accept_rows_kernel(const AcceptParams P)
     // ---- rejected (or bonus row): inverse-CDF draw from max(0, p - q), or from p itself
     bool use_q = !bonus;
     for (int attempt = 0; attempt < 2; ++attempt) {
-        float rr[VPT][4], sj[VPT];  // residual weights of this thread's ids and their sums per group of 4
+        float rr[VPT][4], sj[VPT], incl[VPT];  // residual weights of this thread's ids and their running sums
         {
             float4 q4[VPT];
 #pragma unroll
@@ -418,98 +568,197 @@ __global__ void __launch_bounds__(NT) accept_rows_kernel(const AcceptParams P)
                 rr[j][1] = fmaxf(0.f, x[j][1] * invZ - q4[j].y);
                 rr[j][2] = fmaxf(0.f, x[j][2] * invZ - q4[j].z);
                 rr[j][3] = fmaxf(0.f, x[j][3] * invZ - q4[j].w);
-                sj[j] = ((rr[j][0] + rr[j][1]) + rr[j][2]) + rr[j][3];
             }
         }
-        float incl[VPT];
-#pragma unroll
-        for (int j = 0; j < VPT; ++j) {
-            float v = sj[j];
-#pragma unroll
-            for (int o = 1; o < 32; o <<= 1) {
-                const float up = __shfl_up_sync(0xffffffffu, v, o);
-                if (lane >= o) v += up;
-            }
-            incl[j] = v;
-            if (lane == 31) s_wt[j * NW + warp] = v;
-        }
-        __syncthreads();
-        if (warp == 0) {  // exclusive prefix of the VPT * NW warp totals (ascending id order), by one warp
-            constexpr int E = VPT * NW, PER = (E + 31) / 32;
-            float ent[PER], run = 0.f;
-#pragma unroll
-            for (int t = 0; t < PER; ++t) {
-                ent[t] = lane * PER + t < E ? s_wt[lane * PER + t] : 0.f;
-                run += ent[t];
-            }
-            float incl_l = run;
-#pragma unroll
-            for (int o = 1; o < 32; o <<= 1) {
-                const float up = __shfl_up_sync(0xffffffffu, incl_l, o);
-                if (lane >= o) incl_l += up;
-            }
-            float base = incl_l - run;
-#pragma unroll
-            for (int t = 0; t < PER; ++t) {
-                if (lane * PER + t < E) s_wbase[lane * PER + t] = base;
-                base += ent[t];
-            }
-            if (lane == 31) s_total = incl_l;
-            if (lane == 0) s_tok = 0x7fffffff;
-        }
-        __syncthreads();
-        const float total = s_total;
+        const float total = row_mass<NT, VPT>(rr, sj, incl, sh);
         if (use_q && !(total > 0.f)) {  // p <= q everywhere: draw from p with the same uniform
             use_q = false;
             continue;
         }
-        const float tl = u_res * total;
-        // pass 0: elements where the running sum crosses tl; pass 1 (only if the block-wide sums
-        // disagree at a thread boundary): the first element whose running sum exceeds tl
-        for (int pass = 0; pass < 2; ++pass) {
-#pragma unroll
-            for (int j = 0; j < VPT; ++j) {
-                const float excl = s_wbase[j * NW + warp] + (incl[j] - sj[j]);
-                const bool look = pass == 0 ? (excl <= tl && excl + sj[j] > tl) : (excl + sj[j] > tl);
-                if (look) {
-                    const int e0 = 4 * (j * NT + tid);
-                    const float r0 = rr[j][0], r1 = rr[j][1], r2 = rr[j][2], r3 = rr[j][3];
-                    const float c0 = excl + r0, c1 = excl + (r0 + r1), c2 = excl + ((r0 + r1) + r2);
-                    const float c3 = excl + (((r0 + r1) + r2) + r3);
-                    int hit = -1;  // an id without mass is never drawn
-                    if (r0 > 0.f && c0 > tl) hit = 0;
-                    else if (r1 > 0.f && c1 > tl) hit = 1;
-                    else if (r2 > 0.f && c2 > tl) hit = 2;
-                    else if (r3 > 0.f && c3 > tl) hit = 3;
-                    if (hit >= 0) atomicMin(&s_tok, e0 + hit);
-                }
-            }
-            __syncthreads();
-            if (s_tok != 0x7fffffff) break;
-            __syncthreads();
-        }
-        int tok = s_tok;
-        if (tok == 0x7fffffff) {  // rounding left no running sum above tl: the last id with mass
-            __syncthreads();
-            if (tid == 0) s_tok = -1;
-            __syncthreads();
-#pragma unroll
-            for (int j = 0; j < VPT; ++j) {
-                const int e0 = 4 * (j * NT + tid);
-                if (sj[j] > 0.f) {
-                    int last = -1;
-#pragma unroll
-                    for (int c = 0; c < 4; ++c)
-                        if (rr[j][c] > 0.f) last = e0 + c;
-                    if (last >= 0) atomicMax(&s_tok, last);
-                }
-            }
-            __syncthreads();
-            tok = s_tok;
-        }
+        const int tok = row_search<NT, VPT>(rr, sj, incl, u_res * total, sh);
         if (tid == 0) P.row_out[b * P.rows + i] = tok >= 0 ? P.v_begin + tok : ROW_REJECTED_NO_TOKEN;
         return;
     }
+}
+
+// ------------------------------------------------------------------------------------------------
+// Tree verification (several candidates per depth, each with its own draft distribution; Sec. 4.2,
+// Eq. "recur"): one block per (sequence, tree node).  The block computes the node's target
+// distribution exactly as above and then verifies the node's children in order, keeping the
+// refined target max(0, p - q) un-normalised in registers with its mass as a scalar.  Its verdict is
+// the child that passed, or the correction token drawn from the target as refined by every rejection.
+// Every node is judged, whether or not the walk will reach it; a second kernel follows the verdicts
+// from the root.
+struct TreeParams {
+    const float *logits;        // [2B][N][V]
+    const float *q;             // [B][NQ][V]
+    const int32_t *node_token;  // [B][N]
+    const int32_t *node_q;      // [N]
+    const int32_t *child_begin; // [N + 1]
+    const float *u_acc;         // [B][N]
+    const float *u_res;         // [B][N]
+    int B, N, NQ, V, v_begin, n;
+    float cfg_scale, temperature;
+    int top_k;
+    int vec_ok;
+    int32_t *verdict;  // [B][N]: >= 0 the child that passed; -1 stop without a token; <= -2 stop, token = -v - 2
+    int32_t *dev_status;
+};
+
+template <int NT, int VPT>
+__global__ void __launch_bounds__(NT) tree_rows_kernel(const TreeParams P)
+{
+    __shared__ RowShared<NT, VPT> sh;
+    __shared__ int s_cq[kMaxChildren];
+    const int tid = threadIdx.x;
+    hawk::allow_dependent_launch();
+    hawk::grid_dependency_wait();
+
+    const int row = blockIdx.x;  // node-major
+    const int node = row / P.B, b = row - node * P.B;
+    const int n = P.n;
+    const bool vec_ok = P.vec_ok != 0;
+    const float *lc = P.logits + (static_cast<size_t>(b) * P.N + node) * P.V + P.v_begin;
+    const float *lu = P.logits + (static_cast<size_t>(P.B + b) * P.N + node) * P.V + P.v_begin;
+    int flags = 0;
+
+    // children of the node; ids must grow along the walk so that it ends
+    int cb = P.child_begin[node], ce = P.child_begin[node + 1];
+    if (cb < ce) {
+        const int cb1 = max(node + 1, min(cb, P.N));
+        const int ce1 = max(cb1, min(ce, min(P.N, cb1 + kMaxChildren)));
+        if (cb1 != cb || ce1 != ce) flags |= HAWK_DEV_BAD_TREE;  // clamped: the walk still ends
+        cb = cb1;
+        ce = ce1;
+    } else {  // a leaf (begin == end, whatever the value)
+        if (cb > ce) flags |= HAWK_DEV_BAD_TREE;
+        ce = cb;
+    }
+    const int nc = ce - cb;
+    // this thread's child (threads 0 .. nc-1): token, draft row and uniform, requested before the rows
+    int my_tok = 0, my_q = 0;
+    float my_u = 0.f, my_qx = 0.f;
+    if (tid < nc) {
+        my_tok = P.node_token[b * P.N + cb + tid];
+        my_q = P.node_q[cb + tid];
+        my_u = P.u_acc[b * P.N + cb + tid];
+    }
+    const float u_res = P.u_res[b * P.N + node];
+
+    float x[VPT][4];
+    float mx, mn;
+    int cnt;
+    row_load<NT, VPT>(lc, lu, n, vec_ok, P.cfg_scale, P.temperature, x, mx, mn, cnt, flags);
+
+    if (tid < nc) {
+        if (my_tok < P.v_begin || my_tok >= P.v_begin + n) {
+            flags |= HAWK_DEV_BAD_DRAFT;
+            my_tok = my_tok < P.v_begin ? P.v_begin : P.v_begin + n - 1;
+        }
+        my_tok -= P.v_begin;
+        if (my_q < 0 || my_q >= P.NQ) {
+            flags |= HAWK_DEV_BAD_TREE;
+            my_q = max(0, min(my_q, P.NQ - 1));
+        }
+        my_qx = P.q[(static_cast<size_t>(b) * P.NQ + my_q) * P.V + P.v_begin + my_tok];
+    }
+    if (flags && P.dev_status) atomicOr(P.dev_status, flags);
+
+    block_minmaxcount<NT>(mx, mn, cnt, sh.red);
+    if (cnt == 0) {  // nothing has mass: every candidate is rejected and no token exists
+        if (tid == 0) P.verdict[b * P.N + node] = -1;
+        return;
+    }
+    const float tau = row_topk<NT, VPT>(x, mn, mx, cnt, P.top_k, sh);
+    float mass = row_softmax<NT, VPT>(x, tau, mx, sh);  // x: un-normalised target, p = x / mass
+    if (tid < nc) {  // the children's scalars have long arrived
+        sh.ctok[tid] = my_tok;
+        sh.cqx[tid] = my_qx;
+        sh.cu[tid] = my_u;
+        s_cq[tid] = my_q;
+    }
+    __syncthreads();
+
+    for (int ci = 0; ci < nc; ++ci) {
+        const int xd = sh.ctok[ci];
+        if (tid == ((xd >> 2) % NT)) {  // the thread that holds the candidate's id
+#pragma unroll
+            for (int j = 0; j < VPT; ++j)
+#pragma unroll
+                for (int c = 0; c < 4; ++c)
+                    if (4 * (j * NT + tid) + c == xd) sh.pxe = x[j][c];
+        }
+        __syncthreads();
+        const float px = sh.pxe / mass;
+        const bool accepted = static_cast<double>(sh.cu[ci]) * static_cast<double>(sh.cqx[ci]) < static_cast<double>(px);
+        if (accepted) {
+            if (tid == 0) P.verdict[b * P.N + node] = cb + ci;
+            return;
+        }
+        // rejected: target <- max(0, p - q), kept un-normalised as max(0, x - mass * q)
+        const float *qrow = P.q + (static_cast<size_t>(b) * P.NQ + s_cq[ci]) * P.V + P.v_begin;
+        float rr[VPT][4], rsum = 0.f;
+        {
+            float4 q4[VPT];
+#pragma unroll
+            for (int j = 0; j < VPT; ++j) {
+                const int e0 = 4 * (j * NT + tid);
+                q4[j] = e0 < n ? load4(qrow, e0, n, vec_ok, 0.f) : make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+#pragma unroll
+            for (int j = 0; j < VPT; ++j) {
+                rr[j][0] = fmaxf(0.f, fmaf(-mass, q4[j].x, x[j][0]));
+                rr[j][1] = fmaxf(0.f, fmaf(-mass, q4[j].y, x[j][1]));
+                rr[j][2] = fmaxf(0.f, fmaf(-mass, q4[j].z, x[j][2]));
+                rr[j][3] = fmaxf(0.f, fmaf(-mass, q4[j].w, x[j][3]));
+                rsum += (rr[j][0] + rr[j][1]) + (rr[j][2] + rr[j][3]);
+            }
+        }
+        rsum = block_sum<NT>(rsum, sh.red);
+        if (rsum > 0.f) {  // a residual without mass (p <= q everywhere) leaves the target as it is
+            mass = rsum;
+#pragma unroll
+            for (int j = 0; j < VPT; ++j)
+#pragma unroll
+                for (int c = 0; c < 4; ++c) x[j][c] = rr[j][c];
+        }
+    }
+
+    // ---- every candidate rejected (or a leaf): draw the correction token from the target as refined
+    float sj[VPT], incl[VPT];
+    const float total = row_mass<NT, VPT>(x, sj, incl, sh);
+    int tok = -1;
+    if (total > 0.f) tok = row_search<NT, VPT>(x, sj, incl, u_res * total, sh);
+    if (tid == 0) P.verdict[b * P.N + node] = tok >= 0 ? -(P.v_begin + tok) - 2 : -1;
+}
+
+// One thread per sequence: follows the verdicts from the root.
+__global__ void tree_walk_kernel(const int32_t *verdict, int B, int N, int max_depth, int32_t *accept_len,
+                                 int32_t *out_token, int32_t *path, int32_t *dev_status)
+{
+    hawk::allow_dependent_launch();
+    hawk::grid_dependency_wait();
+    const int b = blockIdx.x * blockDim.x + threadIdx.x;
+    if (b >= B) return;
+    int node = 0, depth = 0, tok = -1;
+    for (int step = 0; step < N; ++step) {
+        const int v = verdict[b * N + node];
+        if (v < 0) {
+            tok = v <= -2 ? -v - 2 : -1;
+            break;
+        }
+        if (v <= node || v >= N) {  // cannot happen with verdicts of tree_rows_kernel; never loop
+            if (dev_status) atomicOr(dev_status, HAWK_DEV_BAD_TREE);
+            break;
+        }
+        if (path && depth < max_depth) path[b * max_depth + depth] = v;
+        ++depth;
+        node = v;
+    }
+    if (path)
+        for (int d = depth; d < max_depth; ++d) path[b * max_depth + d] = -1;
+    accept_len[b] = depth;
+    out_token[b] = tok;
 }
 
 // One thread per sequence: the first rejected row decides accept_len and the correction token.
@@ -542,6 +791,12 @@ template <int NT, int VPT>
 cudaError_t launch_rows(const AcceptParams &P, int grid, cudaStream_t stream)
 {
     return hawk_host::launch_dependent(accept_rows_kernel<NT, VPT>, dim3(grid), dim3(NT), 0, stream, P);
+}
+
+template <int NT, int VPT>
+cudaError_t launch_tree_rows(const TreeParams &P, int grid, cudaStream_t stream)
+{
+    return hawk_host::launch_dependent(tree_rows_kernel<NT, VPT>, dim3(grid), dim3(NT), 0, stream, P);
 }
 
 }  // namespace
@@ -607,6 +862,74 @@ extern "C" hawk_status hawk_cfg_accept(const float *logits, const float *q_probs
     if (err != cudaSuccess) return HAWK_ERR_CUDA;
     err = hawk_host::launch_dependent(accept_finalize_kernel, dim3((B + 127) / 128), dim3(128), 0, st,
                                       static_cast<const int32_t *>(P.row_out), B, K, P.rows, accept_len, out_token);
+    return err == cudaSuccess ? HAWK_OK : HAWK_ERR_CUDA;
+}
+
+
+extern "C" size_t hawk_tree_accept_workspace_bytes(int B, int N)
+{
+    if (B <= 0 || N <= 0) return 0;
+    return static_cast<size_t>(B) * static_cast<size_t>(N) * sizeof(int32_t);
+}
+
+extern "C" hawk_status hawk_tree_accept(const float *logits, const float *q_probs, const int32_t *node_token,
+                                        const int32_t *node_q, const int32_t *child_begin, const float *u_accept,
+                                        const float *u_resample, int B, int N, int NQ, int V, int v_begin,
+                                        int v_end, float cfg_scale, float temperature, int top_k, int max_depth,
+                                        int32_t *accept_len, int32_t *out_token, int32_t *path, void *workspace,
+                                        size_t workspace_bytes, int32_t *dev_status, hawk_stream_t stream)
+{
+    if (B < 0 || N < 0 || NQ < 0 || V < 0 || max_depth < 0) return HAWK_ERR_SHAPE;
+    if (B == 0) return HAWK_OK;
+    if (!logits || !q_probs || !node_token || !node_q || !child_begin || !u_accept || !u_resample || !accept_len ||
+        !out_token)
+        return HAWK_ERR_NULL;
+    if (N < 1 || NQ < 1) return HAWK_ERR_SHAPE;
+    if (v_begin < 0 || v_end > V || v_begin >= v_end) return HAWK_ERR_SHAPE;
+    if (N > 65536) return HAWK_ERR_UNSUPPORTED;
+    const int n = v_end - v_begin;
+    if (n > 32768) return HAWK_ERR_UNSUPPORTED;  // one row must fit one block's registers
+    if (!(temperature == temperature) || !(cfg_scale == cfg_scale) || isinf(temperature) || isinf(cfg_scale))
+        return HAWK_ERR_PARAM;
+    if (!(temperature > 0.f)) return HAWK_ERR_PARAM;
+    if (!hawk_host::aligned16(logits) || !hawk_host::aligned16(q_probs)) return HAWK_ERR_ALIGN;
+    const size_t need = hawk_tree_accept_workspace_bytes(B, N);
+    if (!workspace || workspace_bytes < need) return HAWK_ERR_WORKSPACE;
+    if (!hawk_host::aligned16(workspace)) return HAWK_ERR_ALIGN;
+    if (!hawk_host::is_sm100(nullptr)) return HAWK_ERR_UNSUPPORTED;
+
+    TreeParams P;
+    P.logits = logits;
+    P.q = q_probs;
+    P.node_token = node_token;
+    P.node_q = node_q;
+    P.child_begin = child_begin;
+    P.u_acc = u_accept;
+    P.u_res = u_resample;
+    P.B = B;
+    P.N = N;
+    P.NQ = NQ;
+    P.V = V;
+    P.v_begin = v_begin;
+    P.n = n;
+    P.cfg_scale = cfg_scale;
+    P.temperature = temperature;
+    P.top_k = top_k;
+    P.vec_ok = (V % 4 == 0 && v_begin % 4 == 0) ? 1 : 0;
+    P.verdict = static_cast<int32_t *>(workspace);
+    P.dev_status = dev_status;
+
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    const int grid = B * N;
+    cudaError_t err;
+    if (n <= 4096) err = launch_tree_rows<256, 4>(P, grid, st);
+    else if (n <= 8192) err = launch_tree_rows<512, 4>(P, grid, st);
+    else if (n <= 16384) err = launch_tree_rows<1024, 4>(P, grid, st);
+    else err = launch_tree_rows<1024, 8>(P, grid, st);
+    if (err != cudaSuccess) return HAWK_ERR_CUDA;
+    err = hawk_host::launch_dependent(tree_walk_kernel, dim3((B + 127) / 128), dim3(128), 0, st,
+                                      static_cast<const int32_t *>(P.verdict), B, N, path ? max_depth : 0, accept_len,
+                                      out_token, path, dev_status);
     return err == cudaSuccess ? HAWK_OK : HAWK_ERR_CUDA;
 }
 

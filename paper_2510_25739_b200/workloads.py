@@ -223,3 +223,51 @@ def make_q(cfg: VerifyConfig, seed: int, p: Optional[np.ndarray]) -> np.ndarray:
     if cfg.q_recipe == "mix_row_uniform":
         return mix_q(p, r, row_alphas(cfg, seed))
     raise ValueError(cfg.q_recipe)
+
+
+# ------------------------------------------------------------------------------------------
+# candidate trees (several candidates per depth, Sec. 4.2): topology and draws only
+# ------------------------------------------------------------------------------------------
+def make_tree(branching=(3, 2, 2)) -> dict:
+    """Full tree in breadth-first order with `branching[d]` children under every node of depth d.
+
+    Returns child_begin [N+1], node_depth [N], node_slot [N] (which of its parent's candidates a node
+    is) and node_q [N]: candidate `slot` of depth d draws from draft row d * max(branching) + slot,
+    i.e. every candidate of a level comes from its own draft head.
+    """
+    width = max(branching)
+    depth, slot, level = [0], [0], [0]
+    child_begin = []
+    n = 1
+    for d, c in enumerate(branching):
+        nxt = []
+        for _ in level:
+            child_begin.append(n)
+            for j in range(c):
+                depth.append(d + 1); slot.append(j); nxt.append(n); n += 1
+        level = nxt
+    child_begin += [n] * (len(level) + 1)
+    depth = np.array(depth, np.int32); slot = np.array(slot, np.int32)
+    node_q = np.where(depth > 0, (depth - 1) * width + slot, 0).astype(np.int32)
+    return dict(child_begin=np.array(child_begin, np.int32), node_depth=depth, node_slot=slot, node_q=node_q,
+                N=n, NQ=len(branching) * width)
+
+
+def draw_tree_tokens(q: np.ndarray, tree: dict, seed: int) -> np.ndarray:
+    """node_token[B, N]: one draw per (sequence, depth, candidate slot) from its draft row, shared by all
+    nodes of that depth and slot (the tree is the Cartesian product of the per-position samples)."""
+    rng = np.random.default_rng(seed + 7)
+    B, NQ, V = q.shape
+    u = rng.random((B, NQ))
+    cdf = np.cumsum(q.astype(np.float64), axis=-1)
+    draw = (cdf > (u * cdf[..., -1])[..., None]).argmax(axis=-1).astype(np.int32)     # [B, NQ]
+    tok = draw[:, tree["node_q"]]
+    tok[:, 0] = 0
+    return np.ascontiguousarray(tok)
+
+
+def draw_tree_uniforms(B: int, N: int, seed: int) -> dict:
+    rng = np.random.default_rng(seed + 8)
+    one_below = np.nextafter(np.float32(1.0), np.float32(0.0))
+    return dict(u_accept=np.minimum(rng.random((B, N), dtype=np.float32), one_below),
+                u_resample=np.minimum(rng.random((B, N), dtype=np.float32), one_below))

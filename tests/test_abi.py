@@ -130,3 +130,25 @@ def test_step_host_argument_checks(lib):
     assert lib.hawk_verify_step_host(ctypes.byref(a), None) == OK
     a.B, a.K, a.H, a.D, a.V = 1, 4, 16, 64, 16384
     assert lib.hawk_verify_step_host(ctypes.byref(a), None) == E_NULL     # no buffers given
+
+
+def test_tree_accept_argument_checks(lib):
+    p, odd = ctypes.c_void_p(0x1000), ctypes.c_void_p(0x1004)
+    f = lib.hawk_tree_accept
+
+    def call(lg=p, q=p, tok=p, nq=p, cb=p, ua=p, ur=p, B=2, N=7, NQ=4, V=1024, vb=0, ve=1024, s=3.0, T=1.0, k=100,
+             depth=2, al=p, out=p, path=p, ws=p, wsb=1 << 20):
+        return f(lg, q, tok, nq, cb, ua, ur, B, N, NQ, V, vb, ve, s, T, k, depth, al, out, path, ws, wsb, None, None)
+
+    assert lib.hawk_tree_accept_workspace_bytes(4, 22) == 4 * 22 * 4
+    assert lib.hawk_tree_accept_workspace_bytes(0, 22) == 0
+    assert call(B=0) == OK
+    assert call(B=-1) == E_SHAPE and call(depth=-1) == E_SHAPE
+    assert call(cb=None) == E_NULL and call(out=None) == E_NULL
+    assert call(N=0) == E_SHAPE and call(NQ=0) == E_SHAPE
+    assert call(ve=2000) == E_SHAPE
+    assert call(N=70000) == E_UNSUP
+    assert call(V=40000, ve=40000) == E_UNSUP
+    assert call(T=0.0) == E_PARAM
+    assert call(lg=odd) == E_ALIGN
+    assert call(ws=None) == E_WS and call(wsb=8) == E_WS
