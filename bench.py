@@ -449,6 +449,9 @@ def main():
         "mean_accept_len": mean_len, "sequences_with_rejection": rej, "q_rows_on_chain": q_rows,
     }
 
+    # ---- candidate-tree verification (not part of the timed step): a (3, 2, 2) tree, 22 nodes per sequence
+    stage["tree_accept"] = bench_tree(cfg, stream, torch, hawk, peaks, 1000 * cid + 17 * rank)
+
     # ---- end to end through hawk_verify_step_host: pinned host inputs, copies inside the timed region
     e2e = None
     if not args.no_e2e:
@@ -476,6 +479,61 @@ def main():
         print(json.dumps(line))
     if dist is not None:
         dist.destroy_process_group()
+
+
+def bench_tree(cfg, stream, torch, hawk, peaks, seed, branching=(3, 2, 2)):
+    """Times hawk_tree_accept alone on random logits of the workload's vocabulary (replicas rotating)."""
+    tree = wl.make_tree(branching)
+    N, NQ, B = tree["N"], tree["NQ"], cfg.B
+    dev = torch.device("cuda")
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(seed + 5)
+    row_bytes = cfg.V_valid * 4
+    n_rep = max(2, min(16, -(-3 * L2_BYTES // (2 * B * N * row_bytes))))
+    std = 0.02 * float(np.sqrt(cfg.hidden))
+    child_begin = torch.from_numpy(tree["child_begin"]).to(dev)
+    node_q = torch.from_numpy(tree["node_q"]).to(dev)
+    sets = []
+    for _ in range(n_rep):
+        logits = torch.full((2 * B, N, cfg.V), float("nan"), device=dev)
+        logits[..., cfg.v_begin:cfg.v_end] = std * torch.randn((2 * B, N, cfg.V_valid), generator=gen, device=dev)
+        g = torch.addcmul(logits[B:, 0, cfg.v_begin:cfg.v_end],
+                          logits[:B, 0, cfg.v_begin:cfg.v_end] - logits[B:, 0, cfg.v_begin:cfg.v_end],
+                          torch.tensor(cfg.cfg_scale, device=dev))
+        p0 = torch.softmax(g.double(), dim=-1)[:, None, :]
+        r = torch.softmax(torch.randn((B, NQ, cfg.V_valid), generator=gen, device=dev, dtype=torch.float64), dim=-1)
+        qv = 0.7 * p0 + 0.3 * r
+        q = torch.zeros((B, NQ, cfg.V), device=dev)
+        q[..., cfg.v_begin:cfg.v_end] = qv.float()
+        draw = torch.multinomial(qv.view(-1, cfg.V_valid).float(), 1, generator=gen).view(B, NQ) + cfg.v_begin
+        tok = draw[:, node_q.long()].int().contiguous()
+        ua = torch.rand((B, N), generator=gen, device=dev)
+        ur = torch.rand((B, N), generator=gen, device=dev)
+        sets.append((logits, q, tok, ua, ur))
+    lens = []
+
+    def run(t):
+        a, _, _ = hawk.tree_accept(t[0], t[1], t[2], node_q, child_begin, t[3], t[4], cfg.v_begin, cfg.v_end,
+                                   cfg.cfg_scale, cfg.temperature, cfg.top_k, max_depth=len(branching))
+        return a
+
+    with torch.cuda.stream(stream):
+        for t in sets:
+            lens.append(run(t))
+        stream.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        n = 60
+        e0.record(stream)
+        for i in range(n):
+            run(sets[i % n_rep])
+        e1.record(stream)
+        stream.synchronize()
+    us = e0.elapsed_time(e1) * 1e3 / n
+    nbytes = 2 * B * N * row_bytes
+    return {"us": us, "tree": f"branching {branching}, {N} nodes, {NQ} draft rows per sequence", "rows": B * N,
+            "logit_bytes": nbytes, "GB/s": nbytes / us / 1e3, "frac_hbm": nbytes / us / 1e3 / peaks["hbm_gbs"],
+            "mean_accept_len": float(torch.stack(lens).float().mean().item()),
+            "timing": "eager launches back to back (includes launch overhead), replicas rotating"}
 
 
 def bench_e2e(cfg, reps, stream, torch, hawk, binding, world, dist, steps, warmup):
