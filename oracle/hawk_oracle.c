@@ -19,7 +19,8 @@
  * chi-square of the emitted token, inverse-CDF end points, a hand-computed worked example; for the
  * candidate tree: a hand-computed walk, equality with the chain on chain-shaped trees, chi-square of
  * the first emitted token with three different draft heads, all-rejected rate = prod(1 - alpha_j),
- * candidates drawn from the (refined) target always pass.
+ * candidates drawn from the (refined) target always pass; for tree attention: brute force with a
+ * boolean visibility matrix, chain mask = causal attention, rows off a node's path never reach it.
  * Nothing here is "parity unpinned".
  *
  * OpenMP is used only across independent units (stream x head, token row, sequence).
@@ -420,4 +421,62 @@ int hawk_oracle_tree_accept(const float *logits, const float *q_probs, const int
         free(r);
     }
     return all_flags;
+}
+
+/* ------------------------------------------------------------------------------------------
+ * Step 1 for a candidate tree (Sec. 4.2: "a tree structure is employed to expand the number of
+ * candidates that can be verified simultaneously"; verification is "akin to tree speculative
+ * decoding"): the N tree nodes of a stream are N queries in one forward pass; node i attends to the
+ * whole cached prefix and, inside the block, only to the nodes on its own path from the root.
+ * Plain definition of masked softmax attention:
+ *   key j <  prefix_len[s]                      visible to every node
+ *   key j =  prefix_len[s] + m, 0 <= m < N      visible to node i iff bit m of anc_mask[i] is set
+ * (node i's own key/value row is cache row prefix_len[s] + i; anc_mask[i] has bit i set).
+ * The chain of K drafts is the tree with anc_mask[i] = 2^(i+1) - 1.
+ *   q bf16 [S][N][H][D]; caches bf16 [S][H_kv][L_cap][D]; anc_mask uint32 [N]; out fp64 [S][N][H*D]
+ * ------------------------------------------------------------------------------------------ */
+void hawk_oracle_verify_attn_tree(const uint16_t *q, const uint16_t *k_cache, const uint16_t *v_cache,
+                                  const int32_t *prefix_len, const uint32_t *anc_mask, double *out,
+                                  int S, int N, int H, int H_kv, int D, int L_cap, double sm_scale)
+{
+    int group = H / H_kv;
+#pragma omp parallel for collapse(2) schedule(dynamic)
+    for (int s = 0; s < S; ++s) {
+        for (int h = 0; h < H; ++h) {
+            int hk = h / group;
+            const uint16_t *kb = k_cache + ((size_t)s * H_kv + hk) * (size_t)L_cap * D;
+            const uint16_t *vb = v_cache + ((size_t)s * H_kv + hk) * (size_t)L_cap * D;
+            double *e = (double *)malloc(sizeof(double) * (size_t)(L_cap > 0 ? L_cap : 1));
+            for (int i = 0; i < N; ++i) {
+                int pl = prefix_len[s], n = pl + N;
+                const uint16_t *qv = q + (((size_t)s * N + i) * H + h) * (size_t)D;
+                double m = -INFINITY;
+                for (int j = 0; j < n; ++j) {
+                    int visible = j < pl || ((anc_mask[i] >> (j - pl)) & 1u);
+                    if (!visible) {
+                        e[j] = -INFINITY;
+                        continue;
+                    }
+                    double dot = 0.0;
+                    for (int d = 0; d < D; ++d)
+                        dot += bf16_to_double(qv[d]) * bf16_to_double(kb[(size_t)j * D + d]);
+                    e[j] = sm_scale * dot;
+                    if (e[j] > m) m = e[j];
+                }
+                double z = 0.0;
+                for (int j = 0; j < n; ++j) {
+                    e[j] = isinf(e[j]) ? 0.0 : exp(e[j] - m);
+                    z += e[j];
+                }
+                double *o = out + ((size_t)s * N + i) * (size_t)H * D + (size_t)h * D;
+                for (int d = 0; d < D; ++d) {
+                    double acc = 0.0;
+                    for (int j = 0; j < n; ++j)
+                        if (e[j] != 0.0) acc += e[j] * bf16_to_double(vb[(size_t)j * D + d]);
+                    o[d] = acc / z;
+                }
+            }
+            free(e);
+        }
+    }
 }

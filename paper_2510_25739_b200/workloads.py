@@ -253,6 +253,23 @@ def make_tree(branching=(3, 2, 2)) -> dict:
                 N=n, NQ=len(branching) * width)
 
 
+def tree_ancestor_masks(child_begin: np.ndarray) -> np.ndarray:
+    """anc_mask[i] (uint32): bit m set iff node m lies on the path from the root to node i, i included.
+    Index bookkeeping for the attention mask of a tree with at most 32 nodes."""
+    N = len(child_begin) - 1
+    parent = np.full(N, -1, np.int64)
+    for n in range(N):
+        parent[child_begin[n]:child_begin[n + 1]] = n
+    masks = np.zeros(N, np.uint32)
+    for i in range(N):
+        m, n = 0, i
+        while n >= 0:
+            m |= 1 << n
+            n = parent[n]
+        masks[i] = m
+    return masks
+
+
 def draw_tree_tokens(q: np.ndarray, tree: dict, seed: int) -> np.ndarray:
     """node_token[B, N]: one draw per (sequence, depth, candidate slot) from its draft row, shared by all
     nodes of that depth and slot (the tree is the Cartesian product of the per-position samples)."""
