@@ -78,7 +78,7 @@ int hawk_version(void); /* major*10000 + minor*100 + patch */
  *   workspace    scratch of at least hawk_verify_attn_workspace_bytes(...) bytes, 16-byte aligned;
  *                may be NULL when that function returns 0.  Contents need no initialisation and
  *                are garbage afterwards.
- * Supported: D in {64, 128}; 1 <= K <= 16; H a multiple of H_kv; S*H_kv*L_cap < 2^31.
+ * Supported: D in {64, 128}; 1 <= K <= 32; H a multiple of H_kv; S*H_kv*L_cap < 2^31.
  * Errors: NULL, SHAPE (negative sizes, max_prefix_len + K > L_cap), ALIGN, UNSUPPORTED, WORKSPACE,
  * PARAM (sm_scale not a positive finite number), CUDA.  S == 0 returns HAWK_OK without a launch.
  * ---------------------------------------------------------------------------------------------- */
@@ -88,6 +88,29 @@ hawk_status hawk_verify_attn(const void *q, const void *k_cache, const void *v_c
                              const int32_t *prefix_len, void *out, int S, int K, int H, int H_kv,
                              int D, int L_cap, int max_prefix_len, float sm_scale, void *workspace,
                              size_t workspace_bytes, int32_t *dev_status, hawk_stream_t stream);
+
+/* ------------------------------------------------------------------------------------------------
+ * hawk_verify_attn_tree - the same attention for a candidate tree.
+ *
+ * Operation (Sec. 4.2: the candidates of a tree are verified in one forward pass, "akin to tree
+ * speculative decoding"): the N tree nodes of a stream are N queries; node i attends to the whole
+ * cached prefix and, inside the block, only to the nodes on its own path from the root:
+ *     key j <  prefix_len[s]                  visible to every node
+ *     key j == prefix_len[s] + m, 0 <= m < N  visible to node i iff bit m of anc_mask[i] is set
+ * Node i's own key/value row is cache row prefix_len[s] + i, so anc_mask[i] has bit i set.
+ * hawk_verify_attn is the special case anc_mask[i] = 2^(i+1) - 1.
+ *
+ *   q         bf16 [S][N][H][D]
+ *   anc_mask  uint32 [N], device memory, shared by all streams
+ *   out       bf16 [S][N][H*D]
+ * Everything else, the workspace (hawk_verify_attn_workspace_bytes with K = N) and the errors are
+ * those of hawk_verify_attn; 1 <= N <= 32.
+ * ---------------------------------------------------------------------------------------------- */
+hawk_status hawk_verify_attn_tree(const void *q, const void *k_cache, const void *v_cache,
+                                  const int32_t *prefix_len, const uint32_t *anc_mask, void *out, int S,
+                                  int N, int H, int H_kv, int D, int L_cap, int max_prefix_len,
+                                  float sm_scale, void *workspace, size_t workspace_bytes,
+                                  int32_t *dev_status, hawk_stream_t stream);
 
 /* ------------------------------------------------------------------------------------------------
  * hawk_head_proj - output head: hidden states onto the token codebook.

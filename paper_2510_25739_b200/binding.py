@@ -25,7 +25,7 @@ EXPORTS = (
     "hawk_cfg_accept_workspace_bytes", "hawk_cfg_accept",
     "hawk_verify_step_host",
     "hawk_cfg_accept_noalloc_max_rows", "hawk_cfg_accept_noalloc",
-    "hawk_tree_accept_workspace_bytes", "hawk_tree_accept",
+    "hawk_tree_accept_workspace_bytes", "hawk_tree_accept", "hawk_verify_attn_tree",
 )
 
 
@@ -76,6 +76,8 @@ def load_library() -> ctypes.CDLL:
     lib.hawk_verify_attn_workspace_bytes.argtypes = [i32] * 6
     lib.hawk_verify_attn.restype = i32
     lib.hawk_verify_attn.argtypes = [vp, vp, vp, vp, vp, i32, i32, i32, i32, i32, i32, i32, f32, vp, sz, vp, vp]
+    lib.hawk_verify_attn_tree.restype = i32
+    lib.hawk_verify_attn_tree.argtypes = [vp, vp, vp, vp, vp, vp, i32, i32, i32, i32, i32, i32, i32, f32, vp, sz, vp, vp]
     lib.hawk_head_proj.restype = i32
     lib.hawk_head_proj.argtypes = [vp, vp, vp, i32, i32, i32, i32, i32, vp, vp]
     lib.hawk_cfg_accept_workspace_bytes.restype = sz
@@ -131,8 +133,10 @@ def verify_attn_workspace_bytes(S: int, K: int, H: int, H_kv: int, D: int, max_p
 
 def verify_attn(q: torch.Tensor, k_cache: torch.Tensor, v_cache: torch.Tensor, prefix_len: torch.Tensor,
                 max_prefix_len: int, sm_scale: float, out: Optional[torch.Tensor] = None,
-                workspace: Optional[torch.Tensor] = None, dev_status: Optional[torch.Tensor] = None) -> torch.Tensor:
-    """q [S,K,H,D], caches [S,H_kv,L_cap,D] (bf16), prefix_len [S] int32 -> out [S,K,H*D] bf16."""
+                workspace: Optional[torch.Tensor] = None, dev_status: Optional[torch.Tensor] = None,
+                anc_mask: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """q [S,K,H,D], caches [S,H_kv,L_cap,D] (bf16), prefix_len [S] int32 -> out [S,K,H*D] bf16.
+    With anc_mask (int32 tensor holding the uint32 masks, [K]) the K rows are tree nodes (hawk_verify_attn_tree)."""
     lib = load_library()
     S, K, H, D = q.shape
     _, H_kv, L_cap, _ = k_cache.shape
@@ -147,6 +151,14 @@ def verify_attn(q: torch.Tensor, k_cache: torch.Tensor, v_cache: torch.Tensor, p
     if workspace is None and need:
         workspace = torch.empty(need, dtype=torch.uint8, device=q.device)
     ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    if anc_mask is not None:
+        _check(anc_mask, torch.int32, "anc_mask", (K,))
+        rc = lib.hawk_verify_attn_tree(_ptr(q), _ptr(k_cache), _ptr(v_cache), _ptr(prefix_len), _ptr(anc_mask),
+                                       _ptr(out), S, K, H, H_kv, D, L_cap, int(max_prefix_len), float(sm_scale),
+                                       _ptr(workspace), ws_bytes, _ptr(dev_status), _stream())
+        if rc != 0:
+            raise HawkError(rc, "hawk_verify_attn_tree")
+        return out
     rc = lib.hawk_verify_attn(_ptr(q), _ptr(k_cache), _ptr(v_cache), _ptr(prefix_len), _ptr(out), S, K, H, H_kv, D,
                               L_cap, int(max_prefix_len), float(sm_scale), _ptr(workspace), ws_bytes,
                               _ptr(dev_status), _stream())

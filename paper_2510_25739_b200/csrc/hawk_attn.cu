@@ -53,10 +53,12 @@ struct AttnParams {
     const __nv_bfloat16 *q;
     const int32_t *prefix_len;
     __nv_bfloat16 *out;
-    float *part;  // [workers][2 slots]{o[16 rows][D], (running max in log2 units, running sum)[16 rows]}
+    float *part;  // [workers][2 slots]{o[rows_per_item][D], (running max in log2 units, running sum)[rows_per_item]}
     int S, K, H, H_kv, L_cap;
     int pl_max;           // largest admissible prefix length: min(L_cap - K, max_prefix_len)
-    int chunk_heads;      // query heads handled per item (rows = chunk_heads * K <= 16)
+    const uint32_t *anc_mask;  // [K] block rows visible to each query position; NULL: causal (row i sees rows <= i)
+    int rows_per_item;    // query rows per item, a multiple of 8: the (head of the group, position) pairs of one
+                          // kv head, numbered head-major, are cut into chunks of this many rows
     int chunks;           // items per kv head
     int tiles_per_item;   // tiles of the longest admissible prefix: ceil((max_prefix_len + K) / kTileKeys)
     int workers;          // warps that own a share of the flat tile list
@@ -122,6 +124,13 @@ __device__ __forceinline__ void step(Cursor &c, long long f_end, const AttnParam
     ++c.f;
     ++c.tile;
     if (c.tile == P.tiles_per_item && c.f < f_end) decode_item<TK>(c, P, flags);
+}
+
+// Is the key `rel` rows past the prefix visible to a query whose block-row mask is m?  Prefix keys
+// (rel < 0) always are; block rows past the 32nd never are.
+__device__ __forceinline__ bool key_visible(int rel, uint32_t m)
+{
+    return rel < 0 || (rel < 32 && ((m >> rel) & 1u));
 }
 
 __device__ __forceinline__ uint32_t movmatrix_trans(uint32_t x)
@@ -222,8 +231,8 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const __grid_constant
     uint32_t qb[NQT][DB][2];  // Q^T as the 16 x 8 operand: query row = column tile * 8 + g
     float ot[NQT][DB][4];     // O^T accumulators
     float mrun[NQT][2], lrun[NQT][2];  // running max (log2 units) and this thread's share of the running sum
-    int lim[NQT][2];          // visible keys of the queries in this thread's columns: j < lim
-    int cur_item = -1, h0 = 0, nrows = 0, seg_pl = 0, seg_s = 0;
+    uint32_t qm[NQT][2];      // block rows visible to the queries in this thread's columns (bit m: row prefix + m)
+    int cur_item = -1, hbase = 0, gr0 = 0, nrows = 0, seg_pl = 0, seg_s = 0;
     long long seg_start = 0;
 
     // Writes the finished segment: final bf16 rows if the share held the whole item, else an fp32 partial.
@@ -247,8 +256,8 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const __grid_constant
                 const float inv0 = 1.f / lrun[nq][0], inv1 = 1.f / lrun[nq][1];
                 const int r = nq * 8 + g;  // after the transposes below this thread holds query row r
                 const bool valid = r < nrows;
-                __nv_bfloat16 *dst =
-                    P.out + ((static_cast<size_t>(seg_s) * P.K + r % P.K) * P.H + (h0 + r / P.K)) * D + 2 * tq;
+                __nv_bfloat16 *dst = P.out + ((static_cast<size_t>(seg_s) * P.K + (gr0 + r) % P.K) * P.H +
+                                              (hbase + (gr0 + r) / P.K)) * D + 2 * tq;
 #pragma unroll
                 for (int db = 0; db < DB; ++db) {
                     // (dims g / g+8) x (queries 2tq, 2tq+1)  ->  (query g) x (dims 2tq, 2tq+1 / +8)
@@ -262,7 +271,7 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const __grid_constant
             }
         } else {
             const int slot = seg_start == f_begin ? 0 : 1;
-            float *ps = P.part + (static_cast<size_t>(w) * 2 + slot) * 16 * (D + 2);
+            float *ps = P.part + (static_cast<size_t>(w) * 2 + slot) * P.rows_per_item * (D + 2);
 #pragma unroll
             for (int nq = 0; nq < NQT; ++nq)
 #pragma unroll
@@ -276,7 +285,8 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const __grid_constant
                             pr[db * 16 + 8 + g] = ot[nq][db][2 + c];
                         }
                         if (g == 0)
-                            *reinterpret_cast<float2 *>(ps + 16 * D + 2 * r) = make_float2(mrun[nq][c], lrun[nq][c]);
+                            *reinterpret_cast<float2 *>(ps + P.rows_per_item * D + 2 * r) =
+                                make_float2(mrun[nq][c], lrun[nq][c]);
                     }
                 }
         }
@@ -290,14 +300,14 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const __grid_constant
         const int chunk = it % P.chunks;
         it /= P.chunks;
         const int hk = it % P.H_kv, s = it / P.H_kv;
-        const int hq0 = hk * group + chunk * P.chunk_heads;
-        const int rows = min(P.chunk_heads, group - chunk * P.chunk_heads) * P.K;
+        const int first = chunk * P.rows_per_item;  // first row of the chunk among the kv head's group * K rows
+        const int rows = min(P.rows_per_item, group * P.K - first);
 #pragma unroll
         for (int nq = 0; nq < NQT; ++nq) {
             const int r = nq * 8 + g;  // query row whose values this thread feeds into the operand
             const bool valid = r < rows;
-            const __nv_bfloat16 *qr =
-                P.q + ((static_cast<size_t>(s) * P.K + r % P.K) * P.H + (hq0 + r / P.K)) * D + 2 * tq;
+            const __nv_bfloat16 *qr = P.q + ((static_cast<size_t>(s) * P.K + (first + r) % P.K) * P.H +
+                                             (hk * group + (first + r) / P.K)) * D + 2 * tq;
 #pragma unroll
             for (int kk = 0; kk < DB; ++kk) {
                 dst[nq][kk][0] = valid ? *reinterpret_cast<const uint32_t *>(qr + kk * 16) : 0u;
@@ -320,9 +330,9 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const __grid_constant
             seg_start = cc.f;
             seg_pl = cc.pl;
             seg_s = cc.s;
-            h0 = cc.hk * group + cc.chunk * P.chunk_heads;
-            const int nheads = min(P.chunk_heads, group - cc.chunk * P.chunk_heads);
-            nrows = nheads * P.K;
+            hbase = cc.hk * group;
+            gr0 = cc.chunk * P.rows_per_item;
+            nrows = min(P.rows_per_item, group * P.K - gr0);
             if (qn_item == cc.item) {
 #pragma unroll
                 for (int nq = 0; nq < NQT; ++nq)
@@ -346,7 +356,8 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const __grid_constant
                 for (int c = 0; c < 2; ++c) {
                     mrun[nq][c] = -CUDART_INF_F;
                     lrun[nq][c] = 0.f;
-                    lim[nq][c] = cc.pl + (nq * 8 + 2 * tq + c) % P.K + 1;
+                    const int pos = (gr0 + nq * 8 + 2 * tq + c) % P.K;  // (padding rows get some position's mask)
+                    qm[nq][c] = P.anc_mask ? P.anc_mask[pos] : (2u << pos) - 1u;
                 }
             }
         }
@@ -377,13 +388,13 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const __grid_constant
         if (tile_key0 + TK > pl) {
 #pragma unroll
             for (int kb = 0; kb < KB; ++kb) {
-                const int j0 = tile_key0 + kb * 16 + g, j1 = j0 + 8;
+                const int rel0 = tile_key0 + kb * 16 + g - pl, rel1 = rel0 + 8;
 #pragma unroll
                 for (int nq = 0; nq < NQT; ++nq) {
-                    if (j0 >= lim[nq][0]) sc[nq][kb][0] = -CUDART_INF_F;
-                    if (j0 >= lim[nq][1]) sc[nq][kb][1] = -CUDART_INF_F;
-                    if (j1 >= lim[nq][0]) sc[nq][kb][2] = -CUDART_INF_F;
-                    if (j1 >= lim[nq][1]) sc[nq][kb][3] = -CUDART_INF_F;
+                    if (!key_visible(rel0, qm[nq][0])) sc[nq][kb][0] = -CUDART_INF_F;
+                    if (!key_visible(rel0, qm[nq][1])) sc[nq][kb][1] = -CUDART_INF_F;
+                    if (!key_visible(rel1, qm[nq][0])) sc[nq][kb][2] = -CUDART_INF_F;
+                    if (!key_visible(rel1, qm[nq][1])) sc[nq][kb][3] = -CUDART_INF_F;
                 }
             }
         }
@@ -513,9 +524,8 @@ __global__ void attn_combine_kernel(const AttnParams P, int items, int rows_per_
         it /= P.chunks;
         hk = it % P.H_kv;
         s = it / P.H_kv;
-        const int nheads = min(P.chunk_heads, group - chunk * P.chunk_heads);
         // one share held the whole item and wrote the result itself; rows past the item's last do not exist
-        active = g_first != g_last && r < nheads * P.K;
+        active = g_first != g_last && r < min(P.rows_per_item, group * P.K - chunk * P.rows_per_item);
     }
     // tile offset inside the item at which each contribution starts, and where it is stored
     const float *slot[kAhead];
@@ -525,7 +535,7 @@ __global__ void attn_combine_kernel(const AttnParams P, int items, int rows_per_
         const int gg = min(g_first + t, g_last);
         const long long sb = share_begin(gg, T, P.workers);
         seg_off[t] = static_cast<int>((sb > a ? sb : a) - a);
-        slot[t] = P.part + (static_cast<size_t>(gg) * 2 + (a <= sb ? 0 : 1)) * 16 * (D + 2);
+        slot[t] = P.part + (static_cast<size_t>(gg) * 2 + (a <= sb ? 0 : 1)) * P.rows_per_item * (D + 2);
     }
     grid_dependency_wait();  // every thread waits, so this grid cannot retire before the attention kernel has
     if (!active) return;
@@ -535,7 +545,7 @@ __global__ void attn_combine_kernel(const AttnParams P, int items, int rows_per_
     const int pl_raw = P.prefix_len[s];
 #pragma unroll
     for (int t = 0; t < kAhead; ++t) {  // slots always exist; which of them were written is decided below
-        ml[t] = *reinterpret_cast<const float2 *>(slot[t] + 16 * D + 2 * r);
+        ml[t] = *reinterpret_cast<const float2 *>(slot[t] + P.rows_per_item * D + 2 * r);
         const float *ps = slot[t] + r * D + lane * PER;
         if constexpr (PER == 2) {
             const float2 x = *reinterpret_cast<const float2 *>(ps);
@@ -571,15 +581,16 @@ __global__ void attn_combine_kernel(const AttnParams P, int items, int rows_per_
     for (int gg = g_first + kAhead; gg <= g_last; ++gg) {  // items spread over more shares than that: one by one
         const long long sb = share_begin(gg, T, P.workers);
         if ((sb > a ? sb : a) - a >= ntiles) break;
-        const float *sl = P.part + (static_cast<size_t>(gg) * 2 + (a <= sb ? 0 : 1)) * 16 * (D + 2);
-        const float2 m_l = *reinterpret_cast<const float2 *>(sl + 16 * D + 2 * r);
+        const float *sl = P.part + (static_cast<size_t>(gg) * 2 + (a <= sb ? 0 : 1)) * P.rows_per_item * (D + 2);
+        const float2 m_l = *reinterpret_cast<const float2 *>(sl + P.rows_per_item * D + 2 * r);
         float val[PER];
 #pragma unroll
         for (int c = 0; c < PER; ++c) val[c] = sl[r * D + lane * PER + c];
         fold(m_l, val);
     }
     const float inv = 1.f / ll;
-    const int h = hk * group + chunk * P.chunk_heads + r / P.K, i = r % P.K;
+    const int gr = chunk * P.rows_per_item + r;
+    const int h = hk * group + gr / P.K, i = gr % P.K;
     __nv_bfloat16 *dst = P.out + ((static_cast<size_t>(s) * P.K + i) * P.H + h) * D + lane * PER;
 #pragma unroll
     for (int c = 0; c < PER; c += 2)
@@ -587,7 +598,7 @@ __global__ void attn_combine_kernel(const AttnParams P, int items, int rows_per_
 }
 
 struct AttnPlan {
-    int chunk_heads, chunks, items, rows_per_item, tiles_per_item, workers, grid;
+    int chunks, items, rows_per_item, tiles_per_item, workers, grid;
     long long total_tiles;
     bool any_cut;  // some item's tiles are spread over more than one share: partials + merge kernel needed
 };
@@ -597,10 +608,10 @@ AttnPlan make_plan(int S, int K, int H, int H_kv, int D, int max_prefix_len)
 {
     AttnPlan pl;
     const int group = H / H_kv;
-    pl.chunk_heads = group < 16 / K ? group : 16 / K;
-    if (pl.chunk_heads < 1) pl.chunk_heads = 1;
-    pl.chunks = (group + pl.chunk_heads - 1) / pl.chunk_heads;
-    pl.rows_per_item = pl.chunk_heads * K;
+    const int total_rows = group * K;            // (head of the group, position) pairs sharing one kv head
+    const int rows_max = D == 64 ? 32 : 16;      // what one warp's registers hold
+    pl.chunks = (total_rows + rows_max - 1) / rows_max;
+    pl.rows_per_item = ((total_rows + pl.chunks - 1) / pl.chunks + 7) / 8 * 8;
     pl.items = S * H_kv * pl.chunks;
     const int tk = D == 64 ? AttnCfg<64>::kTileKeys : AttnCfg<128>::kTileKeys;
     pl.tiles_per_item = (max_prefix_len + K + tk - 1) / tk;
@@ -635,23 +646,26 @@ cudaError_t launch_attn(const CUtensorMap &map_k, const CUtensorMap &map_v, cons
 
 extern "C" size_t hawk_verify_attn_workspace_bytes(int S, int K, int H, int H_kv, int D, int max_prefix_len)
 {
-    if (S <= 0 || K < 1 || K > 16 || H <= 0 || H_kv <= 0 || H % H_kv != 0 || (D != 64 && D != 128) ||
+    if (S <= 0 || K < 1 || K > 32 || H <= 0 || H_kv <= 0 || H % H_kv != 0 || (D != 64 && D != 128) ||
         max_prefix_len < 0)
         return 0;
     const AttnPlan pl = make_plan(S, K, H, H_kv, D, max_prefix_len);
     if (!pl.any_cut) return 0;
-    return static_cast<size_t>(pl.workers) * 2 * 16 * (D + 2) * sizeof(float);
+    return static_cast<size_t>(pl.workers) * 2 * pl.rows_per_item * (D + 2) * sizeof(float);
 }
 
-extern "C" hawk_status hawk_verify_attn(const void *q, const void *k_cache, const void *v_cache,
-                                        const int32_t *prefix_len, void *out, int S, int K, int H, int H_kv, int D,
-                                        int L_cap, int max_prefix_len, float sm_scale, void *workspace,
-                                        size_t workspace_bytes, int32_t *dev_status, hawk_stream_t stream)
+namespace {
+
+// Common body of hawk_verify_attn (anc_mask == NULL: causal block) and hawk_verify_attn_tree.
+hawk_status verify_attn_impl(const void *q, const void *k_cache, const void *v_cache, const int32_t *prefix_len,
+                             const uint32_t *anc_mask, void *out, int S, int K, int H, int H_kv, int D, int L_cap,
+                             int max_prefix_len, float sm_scale, void *workspace, size_t workspace_bytes,
+                             int32_t *dev_status, hawk_stream_t stream)
 {
     if (S < 0 || K < 0 || H < 0 || H_kv < 0 || D < 0 || L_cap < 0 || max_prefix_len < 0) return HAWK_ERR_SHAPE;
     if (S == 0) return HAWK_OK;
     if (!q || !k_cache || !v_cache || !prefix_len || !out) return HAWK_ERR_NULL;
-    if (K < 1 || K > 16 || (D != 64 && D != 128) || H < 1 || H_kv < 1 || H % H_kv != 0) return HAWK_ERR_UNSUPPORTED;
+    if (K < 1 || K > 32 || (D != 64 && D != 128) || H < 1 || H_kv < 1 || H % H_kv != 0) return HAWK_ERR_UNSUPPORTED;
     if (max_prefix_len + K > L_cap) return HAWK_ERR_SHAPE;
     if (static_cast<long long>(S) * H_kv * L_cap >= (1ll << 31)) return HAWK_ERR_UNSUPPORTED;
     if (!(sm_scale > 0.f) || isinf(sm_scale)) return HAWK_ERR_PARAM;
@@ -685,7 +699,8 @@ extern "C" hawk_status hawk_verify_attn(const void *q, const void *k_cache, cons
     P.H_kv = H_kv;
     P.L_cap = L_cap;
     P.pl_max = max_prefix_len < L_cap - K ? max_prefix_len : L_cap - K;
-    P.chunk_heads = pl.chunk_heads;
+    P.anc_mask = anc_mask;
+    P.rows_per_item = pl.rows_per_item;
     P.chunks = pl.chunks;
     P.tiles_per_item = pl.tiles_per_item;
     P.workers = pl.workers;
@@ -694,13 +709,17 @@ extern "C" hawk_status hawk_verify_attn(const void *q, const void *k_cache, cons
     P.dev_status = dev_status;
 
     cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
-    const bool wide = pl.rows_per_item > 8;  // more than one 8-query column tile
-    cudaError_t err;
-    if (D == 64)
-        err = wide ? launch_attn<64, 2>(map_k, map_v, P, pl.grid, st) : launch_attn<64, 1>(map_k, map_v, P, pl.grid, st);
-    else
-        err = wide ? launch_attn<128, 2>(map_k, map_v, P, pl.grid, st)
-                   : launch_attn<128, 1>(map_k, map_v, P, pl.grid, st);
+    const int nqt = pl.rows_per_item / 8;  // 8-query column tiles per item: 1..4 (D = 64), 1..2 (D = 128)
+    cudaError_t err = cudaErrorInvalidValue;
+    if (D == 64) {
+        if (nqt == 1) err = launch_attn<64, 1>(map_k, map_v, P, pl.grid, st);
+        else if (nqt == 2) err = launch_attn<64, 2>(map_k, map_v, P, pl.grid, st);
+        else if (nqt == 3) err = launch_attn<64, 3>(map_k, map_v, P, pl.grid, st);
+        else if (nqt == 4) err = launch_attn<64, 4>(map_k, map_v, P, pl.grid, st);
+    } else {
+        if (nqt == 1) err = launch_attn<128, 1>(map_k, map_v, P, pl.grid, st);
+        else if (nqt == 2) err = launch_attn<128, 2>(map_k, map_v, P, pl.grid, st);
+    }
     if (err != cudaSuccess) return HAWK_ERR_CUDA;
     if (pl.any_cut) {
         const int threads = 256;
@@ -713,4 +732,26 @@ extern "C" hawk_status hawk_verify_attn(const void *q, const void *k_cache, cons
         if (err != cudaSuccess) return HAWK_ERR_CUDA;
     }
     return HAWK_OK;
+}
+
+}  // namespace
+
+extern "C" hawk_status hawk_verify_attn(const void *q, const void *k_cache, const void *v_cache,
+                                        const int32_t *prefix_len, void *out, int S, int K, int H, int H_kv, int D,
+                                        int L_cap, int max_prefix_len, float sm_scale, void *workspace,
+                                        size_t workspace_bytes, int32_t *dev_status, hawk_stream_t stream)
+{
+    return verify_attn_impl(q, k_cache, v_cache, prefix_len, nullptr, out, S, K, H, H_kv, D, L_cap, max_prefix_len,
+                            sm_scale, workspace, workspace_bytes, dev_status, stream);
+}
+
+extern "C" hawk_status hawk_verify_attn_tree(const void *q, const void *k_cache, const void *v_cache,
+                                             const int32_t *prefix_len, const uint32_t *anc_mask, void *out, int S,
+                                             int N, int H, int H_kv, int D, int L_cap, int max_prefix_len,
+                                             float sm_scale, void *workspace, size_t workspace_bytes,
+                                             int32_t *dev_status, hawk_stream_t stream)
+{
+    if (S > 0 && !anc_mask) return HAWK_ERR_NULL;
+    return verify_attn_impl(q, k_cache, v_cache, prefix_len, anc_mask, out, S, N, H, H_kv, D, L_cap, max_prefix_len,
+                            sm_scale, workspace, workspace_bytes, dev_status, stream);
 }

@@ -58,7 +58,7 @@ def test_workspace_queries(lib):
     assert lib.hawk_verify_attn_workspace_bytes(0, 4, 16, 16, 64, 128) == 0
     assert lib.hawk_verify_attn_workspace_bytes(2, 4, 16, 16, 96, 128) == 0
     need = lib.hawk_verify_attn_workspace_bytes(16, 5, 20, 20, 64, 1144)
-    assert need > 0 and need % (2 * 16 * 66 * 4) == 0
+    assert need > 0 and need % (2 * 8 * 66 * 4) == 0          # K = 5 rows round up to 8 per item
     # one tile per item and one share per tile: nothing is cut, no workspace
     assert lib.hawk_verify_attn_workspace_bytes(2, 1, 1, 1, 64, 0) == 0
     assert lib.hawk_cfg_accept_workspace_bytes(8, 5, 16384) >= 8 * 5 * 4
@@ -80,7 +80,7 @@ def test_attn_argument_checks(lib):
     assert call(S=-1) == E_SHAPE
     assert call(q=None) == E_NULL
     assert call(out=None) == E_NULL
-    assert call(K=0) == E_UNSUP and call(K=17) == E_UNSUP
+    assert call(K=0) == E_UNSUP and call(K=33) == E_UNSUP
     assert call(D=96) == E_UNSUP
     assert call(H=16, H_kv=3) == E_UNSUP
     assert call(mpl=129) == E_SHAPE                      # prefix + K exceeds the cache capacity
@@ -152,3 +152,12 @@ def test_tree_accept_argument_checks(lib):
     assert call(T=0.0) == E_PARAM
     assert call(lg=odd) == E_ALIGN
     assert call(ws=None) == E_WS and call(wsb=8) == E_WS
+
+
+def test_attn_tree_argument_checks(lib):
+    p = ctypes.c_void_p(0x1000)
+    f = lib.hawk_verify_attn_tree
+    assert f(p, p, p, p, None, p, 2, 7, 4, 4, 64, 100, 90, 0.125, None, 0, None, None) == E_NULL   # no mask
+    assert f(p, p, p, p, p, p, 0, 7, 4, 4, 64, 100, 90, 0.125, None, 0, None, None) == OK
+    assert f(p, p, p, p, p, p, 2, 33, 4, 4, 64, 200, 90, 0.125, None, 0, None, None) == E_UNSUP
+    assert f(p, p, p, p, p, p, 2, 22, 4, 4, 64, 100, 90, 0.125, None, 0, None, None) == E_SHAPE    # 90 + 22 > 100
