@@ -293,6 +293,7 @@ def main():
     ap.add_argument("--impl", default="hawk", choices=["hawk", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--e2e-eager", action="store_true", help="time the end-to-end call eagerly instead of as a graph")
     ap.add_argument("--graph-events", action="store_true",
                     help="also record events around the attention call inside the step graphs (perturbs the step)")
     args = ap.parse_args()
@@ -455,7 +456,8 @@ def main():
     # ---- end to end through hawk_verify_step_host: pinned host inputs, copies inside the timed region
     e2e = None
     if not args.no_e2e:
-        e2e = bench_e2e(cfg, reps, stream, torch, hawk, binding, world, dist, min(K_steps, 2000), W)
+        e2e = bench_e2e(cfg, reps, stream, torch, hawk, binding, world, dist, min(K_steps, 2000), W,
+                        eager=args.e2e_eager)
 
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K_steps, "warmup": W,
@@ -536,7 +538,7 @@ def bench_tree(cfg, stream, torch, hawk, peaks, seed, branching=(3, 2, 2)):
             "timing": "eager launches back to back (includes launch overhead), replicas rotating"}
 
 
-def bench_e2e(cfg, reps, stream, torch, hawk, binding, world, dist, steps, warmup):
+def bench_e2e(cfg, reps, stream, torch, hawk, binding, world, dist, steps, warmup, eager=False):
     """Steps through hawk_verify_step_host with pinned host inputs; returns the e2e object."""
     import ctypes
     n_rep = len(reps)
@@ -568,14 +570,31 @@ def bench_e2e(cfg, reps, stream, torch, hawk, binding, world, dist, steps, warmu
     d2h = 2 * cfg.B * 4
     start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     with torch.cuda.stream(stream):
-        for i in range(warmup):
+        for i in range(max(warmup, n_rep)):      # eager first: the library sets itself up outside any capture
             hawk.verify_step_host(args_list[i % n_rep])
+        stream.synchronize()
+        steps_fn, mode = None, "eager calls"
+        if not eager:
+            try:                                  # the same call captured once per replica, replayed per step
+                graphs = []
+                for a in args_list:
+                    g = torch.cuda.CUDAGraph()
+                    with torch.cuda.graph(g, stream=stream):
+                        hawk.verify_step_host(a)
+                    graphs.append(g)
+                steps_fn, mode = (lambda i: graphs[i % n_rep].replay()), "one CUDA graph replay per step"
+            except Exception as exc:              # capture refused: time the eager calls
+                mode = f"eager calls (graph capture failed: {type(exc).__name__})"
+        if steps_fn is None:
+            steps_fn = lambda i: hawk.verify_step_host(args_list[i % n_rep])
+        for i in range(warmup):
+            steps_fn(i)
         if dist is not None:
             dist.barrier()
         torch.cuda.synchronize()
         start.record(stream)
         for i in range(steps):
-            hawk.verify_step_host(args_list[i % n_rep])
+            steps_fn(i)
         stop.record(stream)
         if dist is not None:
             dist.barrier()
@@ -587,7 +606,8 @@ def bench_e2e(cfg, reps, stream, torch, hawk, binding, world, dist, steps, warmu
         ms = float(t.item())
     return {"value": cfg.B * cfg.K * world / (ms / steps * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
             "d2h_bytes_per_step": d2h, "ms_per_step": ms / steps, "steps": steps,
-            "api": "hawk_verify_step_host (pinned host inputs -> device, 3 kernels, results -> host)"}
+            "api": "hawk_verify_step_host (pinned host inputs -> device, 3 kernels, results -> host)",
+            "launch": mode}
 
 
 if __name__ == "__main__":

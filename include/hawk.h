@@ -257,7 +257,10 @@ hawk_status hawk_cfg_accept_noalloc(const float *logits, const float *q_probs, c
  * hawk_verify_attn, hawk_head_proj, hawk_cfg_accept (contracts above, no bonus row), and
  * device->host copies of accept_len and out_token.  The attention output and the head input are
  * separate tensors: the layers between them (output projection, MLP, norm) are not part of this
- * library, so x is an input of the step like q.  The call returns once everything is queued; the
+ * library, so x is an input of the step like q.  The inputs that only the accept stage reads are
+ * copied on a second stream that the library owns (created by the first call on a device: make that
+ * call outside stream capture), forked from and joined back into `stream` by events, so they travel
+ * while attention and the head projection run.  The call returns once everything is queued; the
  * results are valid after the stream has been synchronised.  Use pinned host memory for the copies
  * to be asynchronous.  The KV cache, the head weight and the prefix lengths are resident device
  * state; all d_* staging and workspaces are device memory owned by the caller.

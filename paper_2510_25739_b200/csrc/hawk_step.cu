@@ -1,7 +1,50 @@
 // hawk_verify_step_host: one whole verify step driven from HOST buffers.
 // Copies the step's inputs to caller-provided device staging, runs the three stages on the stream
 // and copies the two result vectors back; nothing here computes anything itself.
+//
+// The inputs that only the accept stage reads (the draft distributions are 85 % of a step's host
+// bytes) travel on a second, library-owned stream while attention and the head projection run, and
+// join the caller's stream before the accept stage: the step costs max(copies, kernels) instead of
+// their sum.  The fork and join are event dependencies, so the call stays asynchronous and can be
+// captured in a CUDA graph like any other stream work.
+#include <mutex>
+
 #include "hawk_common.cuh"
+
+namespace {
+
+struct SideLane {
+    cudaStream_t stream = nullptr;
+    cudaEvent_t fork = nullptr, join = nullptr;
+};
+
+// One side stream and two events per device, created on the first call on that device (make that
+// call outside stream capture) and kept for the life of the process.
+bool side_lane(SideLane **out)
+{
+    constexpr int kMaxDevices = 64;
+    static SideLane lanes[kMaxDevices];
+    static std::mutex mu;
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return false;
+    std::lock_guard<std::mutex> lock(mu);
+    SideLane &l = lanes[dev];
+    if (!l.stream) {
+        cudaStream_t st = nullptr;
+        cudaEvent_t e0 = nullptr, e1 = nullptr;
+        if (cudaStreamCreateWithFlags(&st, cudaStreamNonBlocking) != cudaSuccess ||
+            cudaEventCreateWithFlags(&e0, cudaEventDisableTiming) != cudaSuccess ||
+            cudaEventCreateWithFlags(&e1, cudaEventDisableTiming) != cudaSuccess)
+            return false;
+        l.stream = st;
+        l.fork = e0;
+        l.join = e1;
+    }
+    *out = &l;
+    return true;
+}
+
+}  // namespace
 
 extern "C" hawk_status hawk_verify_step_host(const hawk_step_host_args *a, hawk_stream_t stream)
 {
@@ -22,24 +65,41 @@ extern "C" hawk_status hawk_verify_step_host(const hawk_step_host_args *a, hawk_
         void *dst;
         const void *src;
         size_t bytes;
-    } in[] = {
+    };
+    // needed by attention and the head projection: on the caller's stream, first
+    const Copy early[] = {
         {a->d_q, a->h_q, static_cast<size_t>(M) * hidden * 2},
         {a->d_x, a->h_x, static_cast<size_t>(M) * hidden * 2},
+    };
+    // needed by the accept stage only: on the side stream, behind everything queued on `stream` so far
+    const Copy late[] = {
         {a->d_q_probs, a->h_q_probs, static_cast<size_t>(a->B) * a->K * a->V * 4},
         {a->d_draft, a->h_draft, static_cast<size_t>(a->B) * a->K * 4},
         {a->d_u_accept, a->h_u_accept, static_cast<size_t>(a->B) * a->K * 4},
         {a->d_u_resample, a->h_u_resample, static_cast<size_t>(a->B) * (a->K + 1) * 4},
     };
-    for (const Copy &c : in)
+    SideLane *lane = nullptr;
+    if (!side_lane(&lane)) return HAWK_ERR_CUDA;
+    if (cudaEventRecord(lane->fork, st) != cudaSuccess || cudaStreamWaitEvent(lane->stream, lane->fork, 0) != cudaSuccess)
+        return HAWK_ERR_CUDA;
+    for (const Copy &c : early)
         if (cudaMemcpyAsync(c.dst, c.src, c.bytes, cudaMemcpyHostToDevice, st) != cudaSuccess) return HAWK_ERR_CUDA;
+    bool late_ok = true;
+    for (const Copy &c : late)
+        late_ok = late_ok && cudaMemcpyAsync(c.dst, c.src, c.bytes, cudaMemcpyHostToDevice, lane->stream) == cudaSuccess;
+    // the join is queued whatever happens below, so that a failed call never leaves the side stream forked
+    // off a capturing stream
+    const bool joined = cudaEventRecord(lane->join, lane->stream) == cudaSuccess;
 
     hawk_status rc = hawk_verify_attn(a->d_q, a->d_k_cache, a->d_v_cache, a->d_prefix_len, a->d_attn_out, S, a->K, a->H,
                                       a->H_kv, a->D, a->L_cap, a->max_prefix_len, a->sm_scale, a->d_attn_workspace,
                                       a->attn_workspace_bytes, a->d_status, stream);
+    if (rc == HAWK_OK)
+        rc = hawk_head_proj(a->d_x, a->d_w, a->d_logits, M, static_cast<int>(hidden), a->V, a->v_begin, a->v_end,
+                            a->d_status, stream);
+    const bool rejoined = joined && cudaStreamWaitEvent(st, lane->join, 0) == cudaSuccess;
     if (rc != HAWK_OK) return rc;
-    rc = hawk_head_proj(a->d_x, a->d_w, a->d_logits, M, static_cast<int>(hidden), a->V, a->v_begin, a->v_end,
-                        a->d_status, stream);
-    if (rc != HAWK_OK) return rc;
+    if (!rejoined || !late_ok) return HAWK_ERR_CUDA;
     rc = hawk_cfg_accept(a->d_logits, a->d_q_probs, a->d_draft, a->d_u_accept, a->d_u_resample, a->B, a->K, a->V,
                          a->v_begin, a->v_end, a->cfg_scale, a->temperature, a->top_k, 0, a->d_accept_len,
                          a->d_out_token, nullptr, a->d_accept_workspace, a->accept_workspace_bytes, a->d_status, stream);
