@@ -45,7 +45,7 @@ L2_BYTES = 126 * 1024 * 1024
 # DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) of one hawk_verify_attn call, attention kernel
 # plus merge kernel, from the ncu capture summarised in profiles/; None where no capture of the
 # current kernels exists for that workload.
-ATTN_TRAFFIC_BYTES = {2: None}
+ATTN_TRAFFIC_BYTES = {2: 94_458_000 + 3_658_000 + 2_044_000}   # attention read + write, merge kernel read
 
 
 def measured_peaks():
