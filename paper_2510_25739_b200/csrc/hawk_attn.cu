@@ -4,7 +4,7 @@
 // The kernel is bound by reading the KV cache once from HBM, so it is organised around keeping
 // that stream of bytes flowing without a gap:
 //   - The work is the flat list of KV tiles (item-major; an item is one (stream, kv head, chunk of
-//     <= 16 query rows), a tile is kTileKeys consecutive keys).  The list is cut into equal contiguous
+//     <= 32 query rows), a tile is kTileKeys consecutive keys).  The list is cut into equal contiguous
 //     shares, one per warp of a persistent grid (one block per SM), so every warp reads the same
 //     number of bytes whatever the shape of the batch and no wave of blocks is ever partly empty.
 //   - Each warp is its own pipeline: lane 0 issues TMA tile loads (128-byte swizzle) into the warp's
@@ -15,6 +15,8 @@
 //     queries on the 8-column operand, so a block of K <= 8 drafts wastes no tensor work and the
 //     per-key softmax work is a quarter of the query-major form.  The tensor pipe is only an ALU
 //     offload here; running max/sum softmax stays in registers (one max reduction per tile).
+//     Which block rows a query sees is a 32-bit mask per query: the causal rule for a chain of
+//     drafts, the ancestor set for a candidate tree (hawk_verify_attn_tree).
 //   - A share that holds all tiles of an item writes bf16 output straight from registers.  A share
 //     that holds only part of an item stores an fp32 partial (o, max, sum) in the workspace, and a
 //     small second kernel merges the partials of every item that was cut.
@@ -140,7 +142,7 @@ __device__ __forceinline__ uint32_t movmatrix_trans(uint32_t x)
     return y;
 }
 
-// NQT = number of 8-query column tiles: 1 when an item has at most 8 query rows, else 2.
+// NQT = number of 8-query column tiles of an item: rows_per_item / 8 (1..4 at D = 64, 1..2 at D = 128).
 template <int D, int NQT>
 __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const __grid_constant__ CUtensorMap map_k,
                                                            const __grid_constant__ CUtensorMap map_v,
