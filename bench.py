@@ -452,6 +452,7 @@ def main():
 
     # ---- candidate-tree verification (not part of the timed step): a (3, 2, 2) tree, 22 nodes per sequence
     stage["tree_accept"] = bench_tree(cfg, stream, torch, hawk, peaks, 1000 * cid + 17 * rank)
+    stage["tree_attn"] = bench_tree_attn(cfg, stream, torch, hawk, peaks, 1000 * cid + 17 * rank)
 
     # ---- end to end through hawk_verify_step_host: pinned host inputs, copies inside the timed region
     e2e = None
@@ -536,6 +537,55 @@ def bench_tree(cfg, stream, torch, hawk, peaks, seed, branching=(3, 2, 2)):
             "logit_bytes": nbytes, "GB/s": nbytes / us / 1e3, "frac_hbm": nbytes / us / 1e3 / peaks["hbm_gbs"],
             "mean_accept_len": float(torch.stack(lens).float().mean().item()),
             "timing": "eager launches back to back (includes launch overhead), replicas rotating"}
+
+
+def bench_tree_attn(cfg, stream, torch, hawk, peaks, seed, branching=(3, 2, 2)):
+    """Times hawk_verify_attn_tree alone: the workload's KV shape with the 22 nodes of a (3, 2, 2) tree as queries."""
+    tree = wl.make_tree(branching)
+    N = tree["N"]
+    masks = torch.from_numpy(wl.tree_ancestor_masks(tree["child_begin"]).view(np.int32)).cuda()
+    dev = torch.device("cuda")
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(seed + 9)
+    S, H, Hkv, D, L = cfg.S, cfg.H, cfg.H_kv, cfg.D, cfg.L
+    kv_bytes = 2 * S * Hkv * (L + N) * D * 2
+    n_rep = max(2, min(8, -(-3 * L2_BYTES // kv_bytes)))
+    bf = torch.bfloat16
+    sets = []
+    for _ in range(n_rep):
+        q = torch.randn((S, N, H, D), generator=gen, device=dev).to(bf)
+        kc = torch.randn((S, Hkv, L + N, D), generator=gen, device=dev).to(bf)
+        vc = torch.randn((S, Hkv, L + N, D), generator=gen, device=dev).to(bf)
+        sets.append((q, kc, vc, torch.empty((S, N, H * D), dtype=bf, device=dev)))
+    pl = torch.full((S,), L, dtype=torch.int32, device=dev)
+    ws = torch.empty(max(16, hawk.verify_attn_workspace_bytes(S, N, H, Hkv, D, L)), dtype=torch.uint8, device=dev)
+    scale = 1.0 / float(np.sqrt(D))
+
+    def run(t):
+        hawk.verify_attn(t[0], t[1], t[2], pl, L, scale, out=t[3], workspace=ws, anc_mask=masks)
+
+    with torch.cuda.stream(stream):
+        for t in sets:
+            run(t)
+        stream.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=stream):
+            for t in sets:
+                run(t)
+        g.replay()
+        stream.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        n = 30
+        e0.record(stream)
+        for _ in range(n):
+            g.replay()
+        e1.record(stream)
+        stream.synchronize()
+    us = e0.elapsed_time(e1) * 1e3 / (n * n_rep)
+    nbytes = kv_bytes + 2 * S * N * H * D * 2
+    return {"us": us, "tree": f"branching {branching}, {N} nodes", "algorithmic_bytes": nbytes,
+            "GB/s": nbytes / us / 1e3, "frac_hbm": nbytes / us / 1e3 / peaks["hbm_gbs"],
+            "timing": "graph of back-to-back calls, replicas rotating"}
 
 
 def bench_e2e(cfg, reps, stream, torch, hawk, binding, world, dist, steps, warmup, eager=False):
