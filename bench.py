@@ -453,6 +453,10 @@ def main():
     # ---- candidate-tree verification (not part of the timed step): a (3, 2, 2) tree, 22 nodes per sequence
     stage["tree_accept"] = bench_tree(cfg, stream, torch, hawk, peaks, 1000 * cid + 17 * rank)
     stage["tree_attn"] = bench_tree_attn(cfg, stream, torch, hawk, peaks, 1000 * cid + 17 * rank)
+    if cid == 2:   # the LlamaGen-XL-shaped workload sweeps the KV length over the image: 120 .. 1144
+        stage["attn_kv_sweep"] = {str(L): bench_tree_attn(replace(cfg, L=L), stream, torch, hawk, peaks,
+                                                          1000 * cid + L, branching=None)
+                                  for L in wl.XL_PREFIX_SWEEP}
 
     # ---- end to end through hawk_verify_step_host: pinned host inputs, copies inside the timed region
     e2e = None
@@ -541,9 +545,12 @@ def bench_tree(cfg, stream, torch, hawk, peaks, seed, branching=(3, 2, 2)):
 
 def bench_tree_attn(cfg, stream, torch, hawk, peaks, seed, branching=(3, 2, 2)):
     """Times hawk_verify_attn_tree alone: the workload's KV shape with the 22 nodes of a (3, 2, 2) tree as queries."""
-    tree = wl.make_tree(branching)
-    N = tree["N"]
-    masks = torch.from_numpy(wl.tree_ancestor_masks(tree["child_begin"]).view(np.int32)).cuda()
+    if branching is None:      # the chain of K drafts (causal block) instead of a tree
+        N, masks = cfg.K, None
+    else:
+        tree = wl.make_tree(branching)
+        N = tree["N"]
+        masks = torch.from_numpy(wl.tree_ancestor_masks(tree["child_begin"]).view(np.int32)).cuda()
     dev = torch.device("cuda")
     gen = torch.Generator(device=dev)
     gen.manual_seed(seed + 9)
@@ -583,7 +590,8 @@ def bench_tree_attn(cfg, stream, torch, hawk, peaks, seed, branching=(3, 2, 2)):
         stream.synchronize()
     us = e0.elapsed_time(e1) * 1e3 / (n * n_rep)
     nbytes = kv_bytes + 2 * S * N * H * D * 2
-    return {"us": us, "tree": f"branching {branching}, {N} nodes", "algorithmic_bytes": nbytes,
+    return {"us": us, "queries": f"tree, branching {branching}, {N} nodes" if branching else f"chain of {N} drafts",
+            "kv_length": L, "algorithmic_bytes": nbytes,
             "GB/s": nbytes / us / 1e3, "frac_hbm": nbytes / us / 1e3 / peaks["hbm_gbs"],
             "timing": "graph of back-to-back calls, replicas rotating"}
 
