@@ -34,9 +34,16 @@ using namespace hawk;
 #ifndef HAWK_ATTN_STAGE_KB
 #define HAWK_ATTN_STAGE_KB 8
 #endif
-constexpr int kWarps = HAWK_ATTN_WARPS;  // independent pipelines per block
-constexpr int kThreads = kWarps * 32;
-constexpr int kStages = 3;               // ring depth of one warp
+// Two launch shapes share one kernel (WARPS independent pipelines per block, STAGES tiles deep each;
+// WARPS * STAGES * 8 KB = 192 KB of shared memory either way):
+//   shares: 8 warps x 3 stages.  The flat tile list is cut into equal shares, items may be cut.
+//   whole : 3 warps x 8 stages.  One warp per item, no item is cut and no merge kernel runs; only a
+//           third of the warps work, so each gets a deeper ring to keep as many bytes in flight.
+//           Taken when the items fit (at most 3 per SM) and an item is short enough for one warp.
+constexpr int kWarpsShares = HAWK_ATTN_WARPS, kStagesShares = 3;
+constexpr int kWarpsWhole = 3, kStagesWhole = 8;
+constexpr int kWholeMaxTiles = 12;       // longest item (in tiles) that one warp takes alone: a lone warp needs
+                                         // 0.75 us per tile, so beyond this the shares (and their merge) win
 constexpr int kStageBytes = HAWK_ATTN_STAGE_KB * 1024;  // K and V tile of one stage
 constexpr int kPlanSms = 148;           // launch shape is planned for the B200's 148 SMs
 
@@ -47,8 +54,10 @@ struct AttnCfg {
     static_assert(kTileKeys % 16 == 0 && kTileKeys >= 16, "a tile is a whole number of 16-key MMA blocks");
     static constexpr int kSubTileBytes = kTileKeys * 128;        // one [keys][64 cols] sub-tile
     static_assert(2 * kHalves * kSubTileBytes == kStageBytes, "stage = K tile + V tile");
-    static constexpr size_t kSmemBytes =
-        1024 /*align slack*/ + static_cast<size_t>(kWarps) * kStages * kStageBytes + kWarps * kStages * sizeof(uint64_t);
+    static constexpr size_t smem_bytes(int warps, int stages)
+    {
+        return 1024 /*align slack*/ + static_cast<size_t>(warps) * stages * kStageBytes + warps * stages * sizeof(uint64_t);
+    }
 };
 
 struct AttnParams {
@@ -143,8 +152,8 @@ __device__ __forceinline__ uint32_t movmatrix_trans(uint32_t x)
 }
 
 // NQT = number of 8-query column tiles of an item: rows_per_item / 8 (1..4 at D = 64, 1..2 at D = 128).
-template <int D, int NQT>
-__global__ void __launch_bounds__(kThreads, 1) attn_kernel(const __grid_constant__ CUtensorMap map_k,
+template <int D, int NQT, int kWarps, int kStages>
+__global__ void __launch_bounds__(kWarps * 32, 1) attn_kernel(const __grid_constant__ CUtensorMap map_k,
                                                            const __grid_constant__ CUtensorMap map_v,
                                                            const AttnParams P)
 {
@@ -167,7 +176,9 @@ __global__ void __launch_bounds__(kThreads, 1) attn_kernel(const __grid_constant
     __syncthreads();  // the only block-wide synchronisation: from here on every warp runs alone
     grid_dependency_wait();
 
-    const int w = blockIdx.x * kWarps + warp;
+    // shares: the warps of a block take neighbouring shares; whole: items are dealt out to the blocks in turn
+    const int w = kWarps == kWarpsWhole ? warp * static_cast<int>(gridDim.x) + static_cast<int>(blockIdx.x)
+                                        : static_cast<int>(blockIdx.x) * kWarps + warp;
     if (w >= P.workers) return;
     uint8_t *ring = smem + warp * kStages * kStageBytes;
     uint64_t *full_bar = bars + warp * kStages;
@@ -601,6 +612,7 @@ __global__ void attn_combine_kernel(const AttnParams P, int items, int rows_per_
 
 struct AttnPlan {
     int chunks, items, rows_per_item, tiles_per_item, workers, grid;
+    bool whole;  // one warp per item (3 warps x 8 stages per block) instead of equal shares (8 x 3)
     long long total_tiles;
     bool any_cut;  // some item's tiles are spread over more than one share: partials + merge kernel needed
 };
@@ -618,9 +630,15 @@ AttnPlan make_plan(int S, int K, int H, int H_kv, int D, int max_prefix_len)
     const int tk = D == 64 ? AttnCfg<64>::kTileKeys : AttnCfg<128>::kTileKeys;
     pl.tiles_per_item = (max_prefix_len + K + tk - 1) / tk;
     pl.total_tiles = static_cast<long long>(pl.items) * pl.tiles_per_item;
-    const long long cap = static_cast<long long>(kPlanSms) * kWarps;
-    pl.workers = static_cast<int>(pl.total_tiles < cap ? pl.total_tiles : cap);
-    pl.grid = (pl.workers + kWarps - 1) / kWarps;
+    pl.whole = pl.items <= kPlanSms * kWarpsWhole && pl.tiles_per_item <= kWholeMaxTiles;
+    if (pl.whole) {
+        pl.workers = pl.items;  // share g = item g
+        pl.grid = pl.items < kPlanSms ? pl.items : kPlanSms;
+    } else {
+        const long long cap = static_cast<long long>(kPlanSms) * kWarpsShares;
+        pl.workers = static_cast<int>(pl.total_tiles < cap ? pl.total_tiles : cap);
+        pl.grid = (pl.workers + kWarpsShares - 1) / kWarpsShares;
+    }
     pl.any_cut = false;
     for (int it = 0; it < pl.items && !pl.any_cut; ++it) {
         const long long a = static_cast<long long>(it) * pl.tiles_per_item, b = a + pl.tiles_per_item;
@@ -629,19 +647,28 @@ AttnPlan make_plan(int S, int K, int H, int H_kv, int D, int max_prefix_len)
     return pl;
 }
 
-template <int D, int NQT>
-cudaError_t launch_attn(const CUtensorMap &map_k, const CUtensorMap &map_v, const AttnParams &P, int grid,
-                        cudaStream_t st)
+template <int D, int NQT, int WARPS, int STAGES>
+cudaError_t launch_attn_shape(const CUtensorMap &map_k, const CUtensorMap &map_v, const AttnParams &P, int grid,
+                              cudaStream_t st)
 {
+    constexpr size_t smem = AttnCfg<D>::smem_bytes(WARPS, STAGES);
     static bool attr_done = false;
     if (!attr_done) {
-        const cudaError_t e = cudaFuncSetAttribute(attn_kernel<D, NQT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                                   static_cast<int>(AttnCfg<D>::kSmemBytes));
+        const cudaError_t e = cudaFuncSetAttribute(attn_kernel<D, NQT, WARPS, STAGES>,
+                                                   cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
         if (e != cudaSuccess) return e;
         attr_done = true;
     }
-    return hawk_host::launch_dependent(attn_kernel<D, NQT>, dim3(grid), dim3(kThreads), AttnCfg<D>::kSmemBytes, st,
-                                       map_k, map_v, P);
+    return hawk_host::launch_dependent(attn_kernel<D, NQT, WARPS, STAGES>, dim3(grid), dim3(WARPS * 32), smem, st, map_k,
+                                       map_v, P);
+}
+
+template <int D, int NQT>
+cudaError_t launch_attn(const CUtensorMap &map_k, const CUtensorMap &map_v, const AttnParams &P, int grid, bool whole,
+                        cudaStream_t st)
+{
+    return whole ? launch_attn_shape<D, NQT, kWarpsWhole, kStagesWhole>(map_k, map_v, P, grid, st)
+                 : launch_attn_shape<D, NQT, kWarpsShares, kStagesShares>(map_k, map_v, P, grid, st);
 }
 
 }  // namespace
@@ -714,13 +741,13 @@ hawk_status verify_attn_impl(const void *q, const void *k_cache, const void *v_c
     const int nqt = pl.rows_per_item / 8;  // 8-query column tiles per item: 1..4 (D = 64), 1..2 (D = 128)
     cudaError_t err = cudaErrorInvalidValue;
     if (D == 64) {
-        if (nqt == 1) err = launch_attn<64, 1>(map_k, map_v, P, pl.grid, st);
-        else if (nqt == 2) err = launch_attn<64, 2>(map_k, map_v, P, pl.grid, st);
-        else if (nqt == 3) err = launch_attn<64, 3>(map_k, map_v, P, pl.grid, st);
-        else if (nqt == 4) err = launch_attn<64, 4>(map_k, map_v, P, pl.grid, st);
+        if (nqt == 1) err = launch_attn<64, 1>(map_k, map_v, P, pl.grid, pl.whole, st);
+        else if (nqt == 2) err = launch_attn<64, 2>(map_k, map_v, P, pl.grid, pl.whole, st);
+        else if (nqt == 3) err = launch_attn<64, 3>(map_k, map_v, P, pl.grid, pl.whole, st);
+        else if (nqt == 4) err = launch_attn<64, 4>(map_k, map_v, P, pl.grid, pl.whole, st);
     } else {
-        if (nqt == 1) err = launch_attn<128, 1>(map_k, map_v, P, pl.grid, st);
-        else if (nqt == 2) err = launch_attn<128, 2>(map_k, map_v, P, pl.grid, st);
+        if (nqt == 1) err = launch_attn<128, 1>(map_k, map_v, P, pl.grid, pl.whole, st);
+        else if (nqt == 2) err = launch_attn<128, 2>(map_k, map_v, P, pl.grid, pl.whole, st);
     }
     if (err != cudaSuccess) return HAWK_ERR_CUDA;
     if (pl.any_cut) {
