@@ -177,40 +177,63 @@ struct RowShared {
 // Reads the conditional and unconditional logit rows once and leaves the guided logits of the block's
 // ids in registers (id of x[j][c]: 4 * (j * NT + tid) + c; ids past n hold -inf); also this thread's
 // max, min and count of finite values.
+// The common case runs without a branch: the guided value is computed for every id and replaced by
+// -inf where an input or the result is not finite; which of those deserve the NONFINITE flag (NaN
+// or +inf, as opposed to a plain -inf mask) is sorted out afterwards, and only by threads that met one.
+// `full` (block-uniform): the row fills the block exactly and is 16-byte aligned, so no id needs a
+// bounds check.
 template <int NT, int VPT>
-__device__ __forceinline__ void row_load(const float *lc, const float *lu, int n, bool vec_ok, float cfg_scale,
-                                         float temperature, float (&x)[VPT][4], float &mx, float &mn, int &cnt,
-                                         int &flags)
+__device__ __forceinline__ void row_load(const float *lc, const float *lu, int n, bool vec_ok, bool full,
+                                         float cfg_scale, float temperature, float (&x)[VPT][4], float &mx,
+                                         float &mn, int &cnt, int &flags)
 {
-    constexpr int NW = NT / 32;
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    (void)lane; (void)warp; (void)NW;
+    const int tid = threadIdx.x;
     const bool unit_T = temperature == 1.0f;
     mx = -CUDART_INF_F, mn = CUDART_INF_F, cnt = 0;
-    {
-        float4 c4[VPT], u4[VPT];
+    float4 c4[VPT], u4[VPT];
+    if (full) {
 #pragma unroll
         for (int j = 0; j < VPT; ++j) {  // all loads in flight before the first use
-            const int e0 = 4 * (j * NT + tid);
-            c4[j] = e0 < n ? load4(lc, e0, n, vec_ok, -CUDART_INF_F) : make_float4(0.f, 0.f, 0.f, 0.f);
-            u4[j] = e0 < n ? load4(lu, e0, n, vec_ok, -CUDART_INF_F) : make_float4(0.f, 0.f, 0.f, 0.f);
+            c4[j] = ld_stream4(lc + 4 * (j * NT + tid));
+            u4[j] = ld_stream4(lu + 4 * (j * NT + tid));
         }
+    } else {
 #pragma unroll
         for (int j = 0; j < VPT; ++j) {
             const int e0 = 4 * (j * NT + tid);
-            int fl = 0;
-            x[j][0] = e0 + 0 < n ? guided(c4[j].x, u4[j].x, cfg_scale, temperature, unit_T, fl) : -CUDART_INF_F;
-            x[j][1] = e0 + 1 < n ? guided(c4[j].y, u4[j].y, cfg_scale, temperature, unit_T, fl) : -CUDART_INF_F;
-            x[j][2] = e0 + 2 < n ? guided(c4[j].z, u4[j].z, cfg_scale, temperature, unit_T, fl) : -CUDART_INF_F;
-            x[j][3] = e0 + 3 < n ? guided(c4[j].w, u4[j].w, cfg_scale, temperature, unit_T, fl) : -CUDART_INF_F;
-            flags |= fl;
+            c4[j] = e0 < n ? load4(lc, e0, n, vec_ok, -CUDART_INF_F) : make_float4(-CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F);
+            u4[j] = e0 < n ? load4(lu, e0, n, vec_ok, -CUDART_INF_F) : c4[j];
+        }
+    }
+    bool odd = false;  // met an id whose inputs or result are not finite
 #pragma unroll
-            for (int c = 0; c < 4; ++c)
-                if (x[j][c] > -CUDART_INF_F) {
-                    mx = fmaxf(mx, x[j][c]);
-                    mn = fminf(mn, x[j][c]);
-                    ++cnt;
-                }
+    for (int j = 0; j < VPT; ++j) {
+        const float cs[4] = {c4[j].x, c4[j].y, c4[j].z, c4[j].w}, us[4] = {u4[j].x, u4[j].y, u4[j].z, u4[j].w};
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+            float r = __fmaf_rn(cfg_scale, __fsub_rn(cs[c], us[c]), us[c]);
+            if (!unit_T) r = __fdiv_rn(r, temperature);
+            const bool ok = (fabsf(cs[c]) < CUDART_INF_F) & (fabsf(us[c]) < CUDART_INF_F) & (fabsf(r) < CUDART_INF_F);
+            odd |= !ok;
+            r = ok ? r : -CUDART_INF_F;
+            x[j][c] = r;
+            mx = fmaxf(mx, r);                          // -inf leaves the maximum alone
+            mn = fminf(mn, ok ? r : CUDART_INF_F);
+            cnt += ok;
+        }
+    }
+    if (odd) {  // rare: read those ids again and look exactly (ids past the row end read as -inf: no flag)
+#pragma unroll 1
+        for (int j = 0; j < VPT; ++j) {
+            const int e0 = 4 * (j * NT + tid);
+            if (e0 >= n) break;
+            const float4 a = load4(lc, e0, n, vec_ok, -CUDART_INF_F), b = load4(lu, e0, n, vec_ok, -CUDART_INF_F);
+            int fl = 0;
+            (void)guided(a.x, b.x, cfg_scale, temperature, unit_T, fl);
+            (void)guided(a.y, b.y, cfg_scale, temperature, unit_T, fl);
+            (void)guided(a.z, b.z, cfg_scale, temperature, unit_T, fl);
+            (void)guided(a.w, b.w, cfg_scale, temperature, unit_T, fl);
+            flags |= fl;
         }
     }
 }
@@ -491,7 +514,7 @@ __global__ void __launch_bounds__(NT) accept_rows_kernel(const AcceptParams P)
     float x[VPT][4];
     float mx, mn;
     int cnt;
-    row_load<NT, VPT>(lc, lu, n, vec_ok, P.cfg_scale, P.temperature, x, mx, mn, cnt, flags);
+    row_load<NT, VPT>(lc, lu, n, vec_ok, vec_ok && n == 4 * NT * VPT, P.cfg_scale, P.temperature, x, mx, mn, cnt, flags);
 
     float qx = 0.f;
     if (!bonus) {
@@ -648,7 +671,7 @@ __global__ void __launch_bounds__(NT) tree_rows_kernel(const TreeParams P)
     float x[VPT][4];
     float mx, mn;
     int cnt;
-    row_load<NT, VPT>(lc, lu, n, vec_ok, P.cfg_scale, P.temperature, x, mx, mn, cnt, flags);
+    row_load<NT, VPT>(lc, lu, n, vec_ok, vec_ok && n == 4 * NT * VPT, P.cfg_scale, P.temperature, x, mx, mn, cnt, flags);
 
     if (tid < nc) {
         if (my_tok < P.v_begin || my_tok >= P.v_begin + n) {
