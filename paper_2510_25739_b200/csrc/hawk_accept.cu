@@ -87,16 +87,22 @@ __device__ __forceinline__ int ordered_int(float v)
 }
 __device__ __forceinline__ float ordered_float(int k) { return __int_as_float(k ^ ((k >> 31) & 0x7fffffff)); }
 
+// Scratch of the block-wide reductions.  Every call site has a slot of its own, so a reduction
+// needs ONE barrier (publish, then read): with 32 warps a barrier costs some 400 cycles, and a
+// second one per call only guarded the reuse of the scratch.
+//   slot 0: range of the row          slot 1: range of a crowded bin (narrowing rounds)
+//   slot 2: softmax sum               slot 3: residual mass of a rejected candidate (tree)
+//   slot 4: bin search
+// Two uses of the same slot are always separated by at least one other barrier.
+constexpr int kRedSlots = 5;
 template <int NT>
 struct Scratch {
-    float f[3][32];
-    int i[32], i2[32], i3[32];
-    float scan[33];
-    int iscan[33];
+    float f[kRedSlots][32];
+    int i[kRedSlots][3][32];
 };
 
 // Block-wide max, min and count: one redux instruction per value and level instead of shuffle trees.
-template <int NT>
+template <int NT, int SLOT>
 __device__ __forceinline__ void block_minmaxcount(float &mx, float &mn, int &cnt, Scratch<NT> &s)
 {
     constexpr int kNW = NT / 32;
@@ -104,54 +110,51 @@ __device__ __forceinline__ void block_minmaxcount(float &mx, float &mn, int &cnt
     int kmn = __reduce_min_sync(0xffffffffu, ordered_int(mn));
     cnt = __reduce_add_sync(0xffffffffu, cnt);
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    __syncthreads();
     if (lane == 0) {
-        s.i[warp] = kmx;
-        s.i2[warp] = kmn;
-        s.i3[warp] = cnt;
+        s.i[SLOT][0][warp] = kmx;
+        s.i[SLOT][1][warp] = kmn;
+        s.i[SLOT][2][warp] = cnt;
     }
     __syncthreads();
-    kmx = __reduce_max_sync(0xffffffffu, lane < kNW ? s.i[lane] : ordered_int(-CUDART_INF_F));
-    kmn = __reduce_min_sync(0xffffffffu, lane < kNW ? s.i2[lane] : ordered_int(CUDART_INF_F));
-    cnt = __reduce_add_sync(0xffffffffu, lane < kNW ? s.i3[lane] : 0);
+    kmx = __reduce_max_sync(0xffffffffu, lane < kNW ? s.i[SLOT][0][lane] : ordered_int(-CUDART_INF_F));
+    kmn = __reduce_min_sync(0xffffffffu, lane < kNW ? s.i[SLOT][1][lane] : ordered_int(CUDART_INF_F));
+    cnt = __reduce_add_sync(0xffffffffu, lane < kNW ? s.i[SLOT][2][lane] : 0);
     mx = ordered_float(kmx);
     mn = ordered_float(kmn);
 }
 
-template <int NT>
+template <int NT, int SLOT>
 __device__ __forceinline__ float block_sum(float v, Scratch<NT> &s)
 {
     constexpr int kNW = NT / 32;
     v = hawk::warp_sum(v);
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    if (lane == 0) s.f[SLOT][warp] = v;
     __syncthreads();
-    if (lane == 0) s.f[0][warp] = v;
-    __syncthreads();
-    v = lane < kNW ? s.f[0][lane] : 0.f;
+    v = lane < kNW ? s.f[SLOT][lane] : 0.f;
     return hawk::warp_sum(v);
 }
 
-// Exclusive prefix sum over the block in thread order; *total receives the block sum.  Two barriers:
-// the warp totals go through shared memory once and every warp scans them for itself.
-template <int NT, class T>
-__device__ __forceinline__ T block_exclusive_scan(T v, T *scratch32, T *total)
+// Exclusive prefix sum of ints over the block in thread order; *total receives the block sum.  The
+// warp totals go through shared memory once and every warp scans them for itself.
+template <int NT, int SLOT>
+__device__ __forceinline__ int block_exclusive_scan(int v, Scratch<NT> &s, int *total)
 {
     constexpr int kNW = NT / 32;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    T incl = v;
+    int incl = v;
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
-        T up = __shfl_up_sync(0xffffffffu, incl, o);
+        const int up = __shfl_up_sync(0xffffffffu, incl, o);
         if (lane >= o) incl += up;
     }
-    __syncthreads();  // earlier readers of scratch32 are done
-    if (lane == 31) scratch32[warp] = incl;
+    if (lane == 31) s.i[SLOT][0][warp] = incl;
     __syncthreads();
-    const T w = lane < kNW ? scratch32[lane] : T(0);
-    T wi = w;
+    const int w = lane < kNW ? s.i[SLOT][0][lane] : 0;
+    int wi = w;
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
-        T up = __shfl_up_sync(0xffffffffu, wi, o);
+        const int up = __shfl_up_sync(0xffffffffu, wi, o);
         if (lane >= o) wi += up;
     }
     *total = __shfl_sync(0xffffffffu, wi, 31);
@@ -168,7 +171,7 @@ struct RowShared {
     Scratch<NT> red;
     float wt[VPT * (NT / 32)];
     float wbase[VPT * (NT / 32)];
-    int bin, above, tok;
+    int bin, above, tok, ncand;
     float tau, pxe, total;
     int ctok[kMaxChildren];
     float cqx[kMaxChildren], cu[kMaxChildren];
@@ -262,6 +265,7 @@ __device__ __forceinline__ float row_topk(const float (&x)[VPT][4], float mn, fl
             const float scale = static_cast<float>(kBins) / (hi - lo);
 #pragma unroll
             for (int t = 0; t < BPT; ++t) sh.hist[t * NT + tid] = 0;
+            if (tid == 0) sh.ncand = 0;
             __syncthreads();
             int bins[VPT][4];  // bin of every value held (-1: outside [lo, hi])
 #pragma unroll
@@ -278,7 +282,7 @@ __device__ __forceinline__ float row_topk(const float (&x)[VPT][4], float mn, fl
 #pragma unroll
             for (int t = 0; t < BPT; ++t) local += sh.hist[tid * BPT + t];
             int total;
-            const int excl = block_exclusive_scan<NT, int>(local, sh.red.iscan, &total);
+            const int excl = block_exclusive_scan<NT, 4>(local, sh.red, &total);
             if (excl < k && k <= excl + local) {  // exactly one thread: one of its bins holds the k-th largest
                 int run = excl;
 #pragma unroll
@@ -295,31 +299,23 @@ __device__ __forceinline__ float row_topk(const float (&x)[VPT][4], float mn, fl
             const int bstar = sh.bin, kk = k - sh.above, C = sh.hist[bstar];
             if (C <= kCandMax) {
                 // rank the members of the bin exactly: the kk-th largest of them is the threshold.
-                // They are compacted into shared memory by a prefix sum over the threads' member counts
-                // (atomics on one counter would serialise).
-                int mine = 0;
+                // They are few (a 1024th of the value range), so gathering them through one shared
+                // counter is cheaper than a block-wide prefix sum (measured).
 #pragma unroll
                 for (int j = 0; j < VPT; ++j)
 #pragma unroll
-                    for (int c = 0; c < 4; ++c) mine += bins[j][c] == bstar;
-                int ctotal;
-                int pos = block_exclusive_scan<NT, int>(mine, sh.red.iscan, &ctotal);
-                if (mine) {
-#pragma unroll
-                    for (int j = 0; j < VPT; ++j)
-#pragma unroll
-                        for (int c = 0; c < 4; ++c)
-                            if (bins[j][c] == bstar) sh.cand[pos++] = x[j][c];
-                }
+                    for (int c = 0; c < 4; ++c)
+                        if (bins[j][c] == bstar) sh.cand[atomicAdd(&sh.ncand, 1)] = x[j][c];
                 __syncthreads();
-                if (C <= 32) {  // the usual case: one warp ranks them with shuffles
+                if (C <= 32) {  // the usual case: one warp ranks them, all 32 exchanges in flight at once
                     if (warp == 0) {
                         const float v = lane < C ? sh.cand[lane] : -CUDART_INF_F;
                         int gt = 0, ge = 0;
-                        for (int m = 0; m < C; ++m) {
-                            const float w = __shfl_sync(0xffffffffu, v, m);
+#pragma unroll 8
+                        for (int m = 0; m < 32; ++m) {
+                            const float w = __shfl_sync(0xffffffffu, v, m);  // lanes >= C hold -inf: never > or >= a member
                             gt += w > v;
-                            ge += w >= v;
+                            ge += (w >= v) & (m < C);
                         }
                         if (lane < C && gt < kk && kk <= ge) sh.tau = v;
                     }
@@ -350,7 +346,7 @@ __device__ __forceinline__ float row_topk(const float (&x)[VPT][4], float mn, fl
                         nmx = fmaxf(nmx, x[j][c]);
                         nmn = fminf(nmn, x[j][c]);
                     }
-            block_minmaxcount<NT>(nmx, nmn, dummy, sh.red);
+            block_minmaxcount<NT, 1>(nmx, nmn, dummy, sh.red);
             lo = nmn;
             hi = nmx;
             k = kk;
@@ -376,7 +372,7 @@ __device__ __forceinline__ float row_softmax(float (&x)[VPT][4], float tau, floa
             x[j][c] = e;
             zsum += e;
         }
-    return block_sum<NT>(zsum, sh.red);
+    return block_sum<NT, 2>(zsum, sh.red);
 }
 
 // Running sums of the non-negative weights rr in ascending id order: sj = sum of each group of 4,
@@ -527,7 +523,7 @@ __global__ void __launch_bounds__(NT) accept_rows_kernel(const AcceptParams P)
     }
     if (flags && P.dev_status) atomicOr(P.dev_status, flags);
 
-    block_minmaxcount<NT>(mx, mn, cnt, sh.red);
+    block_minmaxcount<NT, 0>(mx, mn, cnt, sh.red);
 
     if (cnt == 0) {  // nothing has mass: p == 0 everywhere, the draft is rejected, no token exists
         if (P.p_debug) {
@@ -687,7 +683,7 @@ __global__ void __launch_bounds__(NT) tree_rows_kernel(const TreeParams P)
     }
     if (flags && P.dev_status) atomicOr(P.dev_status, flags);
 
-    block_minmaxcount<NT>(mx, mn, cnt, sh.red);
+    block_minmaxcount<NT, 0>(mx, mn, cnt, sh.red);
     if (cnt == 0) {  // nothing has mass: every candidate is rejected and no token exists
         if (tid == 0) P.verdict[b * P.N + node] = -1;
         return;
@@ -737,7 +733,7 @@ __global__ void __launch_bounds__(NT) tree_rows_kernel(const TreeParams P)
                 rsum += (rr[j][0] + rr[j][1]) + (rr[j][2] + rr[j][3]);
             }
         }
-        rsum = block_sum<NT>(rsum, sh.red);
+        rsum = block_sum<NT, 3>(rsum, sh.red);
         if (rsum > 0.f) {  // a residual without mass (p <= q everywhere) leaves the target as it is
             mass = rsum;
 #pragma unroll
