@@ -151,7 +151,7 @@ __device__ __forceinline__ uint32_t movmatrix_trans(uint32_t x)
     return y;
 }
 
-// NQT = number of 8-query column tiles of an item: rows_per_item / 8 (1..4 at D = 64, 1..2 at D = 128).
+// NQT = number of 8-query column tiles of an item: rows_per_item / 8 (1..4 at D = 64, 1..3 at D = 128).
 template <int D, int NQT, int kWarps, int kStages>
 __global__ void __launch_bounds__(kWarps * 32, 1) attn_kernel(const __grid_constant__ CUtensorMap map_k,
                                                            const __grid_constant__ CUtensorMap map_v,
@@ -623,7 +623,7 @@ AttnPlan make_plan(int S, int K, int H, int H_kv, int D, int max_prefix_len)
     AttnPlan pl;
     const int group = H / H_kv;
     const int total_rows = group * K;            // (head of the group, position) pairs sharing one kv head
-    const int rows_max = D == 64 ? 32 : 16;      // what one warp's registers hold
+    const int rows_max = D == 64 ? 32 : 24;      // what one warp's registers hold
     pl.chunks = (total_rows + rows_max - 1) / rows_max;
     pl.rows_per_item = ((total_rows + pl.chunks - 1) / pl.chunks + 7) / 8 * 8;
     pl.items = S * H_kv * pl.chunks;
@@ -738,7 +738,7 @@ hawk_status verify_attn_impl(const void *q, const void *k_cache, const void *v_c
     P.dev_status = dev_status;
 
     cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
-    const int nqt = pl.rows_per_item / 8;  // 8-query column tiles per item: 1..4 (D = 64), 1..2 (D = 128)
+    const int nqt = pl.rows_per_item / 8;  // 8-query column tiles per item: 1..4 (D = 64), 1..3 (D = 128)
     cudaError_t err = cudaErrorInvalidValue;
     if (D == 64) {
         if (nqt == 1) err = launch_attn<64, 1>(map_k, map_v, P, pl.grid, pl.whole, st);
@@ -748,6 +748,7 @@ hawk_status verify_attn_impl(const void *q, const void *k_cache, const void *v_c
     } else {
         if (nqt == 1) err = launch_attn<128, 1>(map_k, map_v, P, pl.grid, pl.whole, st);
         else if (nqt == 2) err = launch_attn<128, 2>(map_k, map_v, P, pl.grid, pl.whole, st);
+        else if (nqt == 3) err = launch_attn<128, 3>(map_k, map_v, P, pl.grid, pl.whole, st);
     }
     if (err != cudaSuccess) return HAWK_ERR_CUDA;
     if (pl.any_cut) {
