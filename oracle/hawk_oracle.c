@@ -21,6 +21,8 @@
  * the first emitted token with three different draft heads, all-rejected rate = prod(1 - alpha_j),
  * candidates drawn from the (refined) target always pass; for tree attention: brute force with a
  * boolean visibility matrix, chain mask = causal attention, rows off a node's path never reach it.
+ * For the draw of the candidates from the pool: point mass, a boundary straddled from both sides, no
+ * mass inside the valid ids, uniform closed form, both end points, chi-square against the row.
  * Nothing here is "parity unpinned".
  *
  * OpenMP is used only across independent units (stream x head, token row, sequence).
@@ -478,5 +480,34 @@ void hawk_oracle_verify_attn_tree(const uint16_t *q, const uint16_t *k_cache, co
             }
             free(e);
         }
+    }
+}
+
+/* ------------------------------------------------------------------------------------------
+ * Candidates from the spatial sampling pool (Sec. 4.2, "Spatial Sampling Pool": the candidate
+ * tree is built from the sampling results of the pool's distributions at each speculation
+ * position): one draw per pool distribution, by inverse CDF in ascending id over the valid ids,
+ * negative or NaN weights counting as zero.  A row without mass yields -1.
+ *   pool_q fp32 [R][V]; u fp32 [R]; row_token int32 [R]; margin fp64 [R] or NULL
+ * ------------------------------------------------------------------------------------------ */
+void hawk_oracle_pool_sample(const float *pool_q, const float *u, int R, int V, int v_begin, int v_end,
+                             int32_t *row_token, double *margin)
+{
+#pragma omp parallel for schedule(dynamic)
+    for (int r = 0; r < R; ++r) {
+        double *w = (double *)calloc((size_t)V, sizeof(double));
+        double total = 0.0;
+        for (int v = v_begin; v < v_end; ++v) {
+            double x = (double)pool_q[(size_t)r * V + v];
+            w[v] = x > 0.0 ? x : 0.0;
+            total += w[v];
+        }
+        if (total > 0.0)
+            row_token[r] = inverse_cdf(w, v_begin, v_end, (double)u[r], total, margin ? &margin[r] : NULL);
+        else {
+            row_token[r] = -1;
+            if (margin) margin[r] = 1.0;
+        }
+        free(w);
     }
 }
