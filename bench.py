@@ -454,6 +454,7 @@ def main():
     # ---- candidate-tree verification (not part of the timed step): a (3, 2, 2) tree, 22 nodes per sequence
     stage["tree_accept"] = bench_tree(cfg, stream, torch, hawk, peaks, 1000 * cid + 17 * rank)
     stage["tree_attn"] = bench_tree_attn(cfg, stream, torch, hawk, peaks, 1000 * cid + 17 * rank)
+    stage["pool"] = bench_pool(cfg, stream, torch, hawk, peaks, 1000 * cid + 17 * rank)
     if cid == 2:   # the LlamaGen-XL-shaped workload sweeps the KV length over the image: 120 .. 1144
         stage["attn_kv_sweep"] = {str(L): bench_tree_attn(replace(cfg, L=L), stream, torch, hawk, peaks,
                                                           1000 * cid + L, branching=None)
@@ -542,6 +543,64 @@ def bench_tree(cfg, stream, torch, hawk, peaks, seed, branching=(3, 2, 2)):
             "logit_bytes": nbytes, "GB/s": nbytes / us / 1e3, "frac_hbm": nbytes / us / 1e3 / peaks["hbm_gbs"],
             "mean_accept_len": float(torch.stack(lens).float().mean().item()),
             "timing": "eager launches back to back (includes launch overhead), replicas rotating"}
+
+
+def bench_pool(cfg, stream, torch, hawk, peaks, seed, IW=32, VSD=2, K=3, branching=(3, 2, 2)):
+    """Times the drafting-side bookkeeping that feeds the tree verification: cache put, pool build, candidate draw
+    (32 x 32 token image, two vertical depths, three horizontal offsets: the 9 draft rows of the (3, 2, 2) tree)."""
+    tree = wl.make_tree(branching)
+    B, N, NQ = cfg.B, tree["N"], K * (1 + VSD)
+    assert tree["NQ"] == NQ
+    dev = torch.device("cuda")
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(seed + 9)
+    node_q = torch.from_numpy(tree["node_q"]).to(dev)
+    row_bytes = cfg.V * 4
+    n_rep = max(2, min(16, -(-3 * L2_BYTES // (2 * B * NQ * row_bytes))))
+
+    def probs(rows):
+        z = torch.zeros((B, rows, cfg.V), device=dev)
+        z[..., cfg.v_begin:cfg.v_end] = torch.softmax(
+            4.0 * torch.randn((B, rows, cfg.V_valid), generator=gen, device=dev), dim=-1)
+        return z
+
+    sets = [(probs(VSD), probs(K), torch.rand((B, NQ), generator=gen, device=dev)) for _ in range(n_rep)]
+    rows, tags = hawk.spec_cache_new(B, IW, VSD, cfg.V)
+    base = 2 * IW + 3
+    with torch.cuda.stream(stream):
+        for T in range(base + n_rep + 1):        # a step at every position so far: every lookup finds its row
+            hawk.spec_cache_put(sets[T % n_rep][0], torch.full((B,), T, dtype=torch.int32, device=dev), rows, tags, IW)
+        pos = [torch.full((B,), base + i, dtype=torch.int32, device=dev) for i in range(n_rep)]
+        pools = [hawk.pool_build(sets[i][1], rows, tags, pos[i], IW, VSD)[0] for i in range(n_rep)]
+        stream.synchronize()
+
+        def timed(fn, n=50):
+            """us per call: one CUDA graph holding the call for every replica, replayed n times."""
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=stream):
+                for i in range(n_rep):
+                    fn(i)
+            for _ in range(3):
+                g.replay()
+            stream.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            for _ in range(n):
+                g.replay()
+            e1.record(stream)
+            stream.synchronize()
+            return e0.elapsed_time(e1) * 1e3 / (n * n_rep)
+
+        us_put = timed(lambda i: hawk.spec_cache_put(sets[i][0], pos[i], rows, tags, IW))
+        us_build = timed(lambda i: hawk.pool_build(sets[i][1], rows, tags, pos[i], IW, VSD, with_source=False))
+        us_sample = timed(lambda i: hawk.pool_sample(pools[i], sets[i][2], node_q, cfg.v_begin, cfg.v_end))
+    b_put, b_build, b_sample = 2 * B * VSD * row_bytes, 2 * B * NQ * row_bytes, B * NQ * cfg.V_valid * 4
+    leg = lambda us, nb: {"us": us, "bytes": nb, "GB/s": nb / us / 1e3, "frac_hbm": nb / us / 1e3 / peaks["hbm_gbs"]}
+    return {"shape": f"IW {IW}, VSD {VSD}, K {K}: {NQ} pool rows and {N} tree nodes per sequence, "
+                     f"cache {hawk.spec_cache_slots(IW, VSD)} rows per sequence",
+            "cache_put": leg(us_put, b_put), "pool_build": leg(us_build, b_build),
+            "pool_sample": leg(us_sample, b_sample),
+            "timing": "each call alone in a CUDA graph over rotating replicas"}
 
 
 def bench_tree_attn(cfg, stream, torch, hawk, peaks, seed, branching=(3, 2, 2)):

@@ -10,6 +10,7 @@
  *   hawk_cfg_accept   guidance combine, temperature, top-k, softmax and speculative rejection
  *                     sampling, returning the accepted length and the correction token;
  *   hawk_tree_accept  the same for a candidate tree with several candidates per depth.
+ *   hawk_spec_cache_*, hawk_pool_*  the cache of vertical predictions and the sampling pool that feed it.
  *
  * Conventions common to all entry points
  *   - Every pointer is a DEVICE pointer owned by the caller unless the comment says "host".  The
@@ -218,6 +219,70 @@ hawk_status hawk_tree_accept(const float *logits, const float *q_probs, const in
                              const float *u_resample, int B, int N, int NQ, int V, int v_begin, int v_end,
                              float cfg_scale, float temperature, int top_k, int max_depth,
                              int32_t *accept_len, int32_t *out_token, int32_t *path, void *workspace,
+                             size_t workspace_bytes, int32_t *dev_status, hawk_stream_t stream);
+
+/* ------------------------------------------------------------------------------------------------
+ * Speculation cache and spatial sampling pool (Sec. 4.2, "Dual Direction Drafting Heads" and "Spatial
+ * Sampling Pool", Eqs. 1-5): the step that hands hawk_tree_accept its draft distributions and tokens.
+ *
+ * Eq. 1: the vertical draft head of depth d (1 <= d <= VSD), run at raster position T of an image IW
+ * tokens wide, predicts the token at T + IW * d.  Eq. 2: those predictions wait in a cache of
+ * IW * VSD * (VSD + 1) / 2 rows per sequence until decoding reaches their target.  Eqs. 3-5: the pool
+ * of speculation point T + n is the horizontal head's distribution for T + n followed, for
+ * dv = 1 .. VSD, by the cached depth-dv prediction made at T + n - IW * dv.
+ *
+ * Device layout, owned by the caller, B sequences:
+ *   cache_rows  fp32  [B][slots][V]   slots = hawk_spec_cache_slots(IW, VSD)
+ *   cache_tags  int32 [B][slots]      raster position that wrote the slot, -1 = never written
+ * hawk_spec_cache_slot gives the slot of the depth-d prediction made at `position`: predictions of one
+ * image column and depth that are alive at the same time come from d consecutive rows, so the row
+ * modulo d tells them apart.  Positions of a sequence must not decrease between calls (a new image
+ * starts with hawk_spec_cache_clear).  A lookup whose slot carries another position finds nothing: no
+ * forward pass started there (the position was accepted inside a step) or it lies above the image.
+ *
+ * hawk_spec_cache_slots    slots per sequence (Eq. 2); 0 if IW < 1 or VSD < 1.  Host only.
+ * hawk_spec_cache_slot     slot index as above, -1 for arguments out of range.  Host only.
+ * hawk_spec_cache_clear    marks every slot of B sequences unwritten.
+ * hawk_spec_cache_put      stores q_vert fp32 [B][VSD][V] (row d-1 = depth d) made at position[b]
+ *                          (int32 [B], device; a negative position stores nothing for that sequence).
+ * hawk_pool_build          q_horiz fp32 [B][K][V] (row n-1 = the horizontal distribution for T + n),
+ *                          position int32 [B] (T of every sequence) ->
+ *                          pool_q fp32 [B][K*(1+VSD)][V], row (n-1)*(1+VSD) + j: j = 0 horizontal,
+ *                          j = dv >= 1 the cached vertical prediction, or a copy of the horizontal row
+ *                          where none is cached; pool_source int32 [B][K*(1+VSD)] (may be NULL): 0, dv,
+ *                          or -dv for the stand-in.  pool_q is laid out as hawk_tree_accept's q_probs
+ *                          with NQ = K*(1+VSD).
+ * hawk_pool_sample         draws one token per pool row by inverse CDF in ascending id over
+ *                          [v_begin, v_end) with u fp32 [B][NQ] in [0,1) (negative weights count as
+ *                          zero; a row without mass gives -1), then fills
+ *                          node_token int32 [B][N]: node_token[b][i] = draw of row node_q[i]
+ *                          (node_q int32 [N], device, as in hawk_tree_accept; the root, i = 0, gets 0).
+ *                          The candidate tree is the Cartesian product of the per-position draws, so
+ *                          all nodes that stand for one pool row carry the same token.  A node_q entry
+ *                          outside [0, NQ) is clamped and flagged HAWK_DEV_BAD_TREE in *dev_status.
+ *                          workspace: hawk_pool_sample_workspace_bytes(B, NQ) bytes, 16-byte aligned.
+ * All pointers are device pointers unless stated; rows are copied with 16-byte accesses when V % 4 == 0
+ * and the buffers are 16-byte aligned, element by element otherwise.  Limits: VSD <= 8; the valid id
+ * range of hawk_pool_sample at most 32768 wide.  Launches are asynchronous on `stream`.
+ * Errors: NULL, SHAPE, ALIGN, UNSUPPORTED, WORKSPACE, CUDA.  B == 0 (or K == 0) returns HAWK_OK.
+ * ---------------------------------------------------------------------------------------------- */
+int hawk_spec_cache_slots(int IW, int VSD);
+
+int hawk_spec_cache_slot(int IW, int VSD, int position, int depth);
+
+hawk_status hawk_spec_cache_clear(int32_t *cache_tags, int B, int IW, int VSD, hawk_stream_t stream);
+
+hawk_status hawk_spec_cache_put(const float *q_vert, const int32_t *position, float *cache_rows,
+                                int32_t *cache_tags, int B, int IW, int VSD, int V, hawk_stream_t stream);
+
+hawk_status hawk_pool_build(const float *q_horiz, const float *cache_rows, const int32_t *cache_tags,
+                            const int32_t *position, float *pool_q, int32_t *pool_source, int B, int K, int IW,
+                            int VSD, int V, hawk_stream_t stream);
+
+size_t hawk_pool_sample_workspace_bytes(int B, int NQ);
+
+hawk_status hawk_pool_sample(const float *pool_q, const float *u, const int32_t *node_q, int32_t *node_token,
+                             int B, int NQ, int N, int V, int v_begin, int v_end, void *workspace,
                              size_t workspace_bytes, int32_t *dev_status, hawk_stream_t stream);
 
 /* ------------------------------------------------------------------------------------------------

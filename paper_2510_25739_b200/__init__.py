@@ -12,7 +12,9 @@ _BINDING_NAMES = (
     "verify_attn", "verify_attn_workspace_bytes", "head_proj",
     "cfg_accept", "cfg_accept_workspace_bytes",
     "verify_step_host", "StepHostArgs",
-    "cfg_accept_noalloc", "cfg_accept_noalloc_max_rows", "tree_accept",
+    "cfg_accept_noalloc", "cfg_accept_noalloc_max_rows", "tree_accept", "verify_attn_tree",
+    "spec_cache_slots", "spec_cache_slot", "spec_cache_new", "spec_cache_clear", "spec_cache_put",
+    "pool_build", "pool_sample", "pool_sample_workspace_bytes",
 )
 
 

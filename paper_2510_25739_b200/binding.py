@@ -26,6 +26,8 @@ EXPORTS = (
     "hawk_verify_step_host",
     "hawk_cfg_accept_noalloc_max_rows", "hawk_cfg_accept_noalloc",
     "hawk_tree_accept_workspace_bytes", "hawk_tree_accept", "hawk_verify_attn_tree",
+    "hawk_spec_cache_slots", "hawk_spec_cache_slot", "hawk_spec_cache_clear", "hawk_spec_cache_put",
+    "hawk_pool_build", "hawk_pool_sample_workspace_bytes", "hawk_pool_sample",
 )
 
 
@@ -94,6 +96,20 @@ def load_library() -> ctypes.CDLL:
     lib.hawk_tree_accept_workspace_bytes.argtypes = [i32, i32]
     lib.hawk_tree_accept.restype = i32
     lib.hawk_tree_accept.argtypes = [vp] * 7 + [i32] * 6 + [f32, f32, i32, i32] + [vp, vp, vp, vp, sz, vp, vp]
+    lib.hawk_spec_cache_slots.restype = i32
+    lib.hawk_spec_cache_slots.argtypes = [i32, i32]
+    lib.hawk_spec_cache_slot.restype = i32
+    lib.hawk_spec_cache_slot.argtypes = [i32, i32, i32, i32]
+    lib.hawk_spec_cache_clear.restype = i32
+    lib.hawk_spec_cache_clear.argtypes = [vp, i32, i32, i32, vp]
+    lib.hawk_spec_cache_put.restype = i32
+    lib.hawk_spec_cache_put.argtypes = [vp, vp, vp, vp, i32, i32, i32, i32, vp]
+    lib.hawk_pool_build.restype = i32
+    lib.hawk_pool_build.argtypes = [vp] * 6 + [i32] * 5 + [vp]
+    lib.hawk_pool_sample_workspace_bytes.restype = sz
+    lib.hawk_pool_sample_workspace_bytes.argtypes = [i32, i32]
+    lib.hawk_pool_sample.restype = i32
+    lib.hawk_pool_sample.argtypes = [vp] * 4 + [i32] * 6 + [vp, sz, vp, vp]
     lib.hawk_verify_step_host.restype = i32
     lib.hawk_verify_step_host.argtypes = [ctypes.POINTER(StepHostArgs), vp]
     _lib = lib
@@ -165,6 +181,12 @@ def verify_attn(q: torch.Tensor, k_cache: torch.Tensor, v_cache: torch.Tensor, p
     if rc != 0:
         raise HawkError(rc, "hawk_verify_attn")
     return out
+
+
+def verify_attn_tree(q: torch.Tensor, k_cache: torch.Tensor, v_cache: torch.Tensor, prefix_len: torch.Tensor,
+                     anc_mask: torch.Tensor, max_prefix_len: int, sm_scale: float, **kwargs) -> torch.Tensor:
+    """hawk_verify_attn_tree: the N rows of q are tree nodes, anc_mask [N] their ancestor bit masks."""
+    return verify_attn(q, k_cache, v_cache, prefix_len, max_prefix_len, sm_scale, anc_mask=anc_mask, **kwargs)
 
 
 def head_proj(x: torch.Tensor, w: torch.Tensor, v_begin: int = 0, v_end: Optional[int] = None,
@@ -287,6 +309,89 @@ def tree_accept(logits: torch.Tensor, q_probs: torch.Tensor, node_token: torch.T
     if rc != 0:
         raise HawkError(rc, "hawk_tree_accept")
     return accept_len, out_token, path
+
+
+def spec_cache_slots(IW: int, VSD: int) -> int:
+    """Rows of the speculation cache per sequence, IW * VSD * (VSD + 1) / 2."""
+    return int(load_library().hawk_spec_cache_slots(int(IW), int(VSD)))
+
+
+def spec_cache_slot(IW: int, VSD: int, position: int, depth: int) -> int:
+    return int(load_library().hawk_spec_cache_slot(int(IW), int(VSD), int(position), int(depth)))
+
+
+def spec_cache_new(B: int, IW: int, VSD: int, V: int, device="cuda"):
+    """Allocates (cache_rows [B,slots,V] fp32, cache_tags [B,slots] int32) and marks every slot unwritten."""
+    slots = spec_cache_slots(IW, VSD)
+    rows = torch.empty((B, slots, V), dtype=torch.float32, device=device)
+    tags = torch.empty((B, slots), dtype=torch.int32, device=device)
+    spec_cache_clear(tags, IW, VSD)
+    return rows, tags
+
+
+def spec_cache_clear(cache_tags: torch.Tensor, IW: int, VSD: int) -> None:
+    B = cache_tags.shape[0]
+    _check(cache_tags, torch.int32, "cache_tags", (B, spec_cache_slots(IW, VSD)))
+    rc = load_library().hawk_spec_cache_clear(_ptr(cache_tags), B, int(IW), int(VSD), _stream())
+    if rc != 0:
+        raise HawkError(rc, "hawk_spec_cache_clear")
+
+
+def spec_cache_put(q_vert: torch.Tensor, position: torch.Tensor, cache_rows: torch.Tensor,
+                   cache_tags: torch.Tensor, IW: int) -> None:
+    """Stores the vertical predictions q_vert [B,VSD,V] made at position [B] into the cache."""
+    B, VSD, V = q_vert.shape
+    slots = spec_cache_slots(IW, VSD)
+    _check(q_vert, torch.float32, "q_vert")
+    _check(position, torch.int32, "position", (B,))
+    _check(cache_rows, torch.float32, "cache_rows", (B, slots, V))
+    _check(cache_tags, torch.int32, "cache_tags", (B, slots))
+    rc = load_library().hawk_spec_cache_put(_ptr(q_vert), _ptr(position), _ptr(cache_rows), _ptr(cache_tags), B,
+                                            int(IW), VSD, V, _stream())
+    if rc != 0:
+        raise HawkError(rc, "hawk_spec_cache_put")
+
+
+def pool_build(q_horiz: torch.Tensor, cache_rows: torch.Tensor, cache_tags: torch.Tensor, position: torch.Tensor,
+               IW: int, VSD: int, with_source: bool = True):
+    """q_horiz [B,K,V] + cache -> (pool_q [B,K*(1+VSD),V], pool_source [B,K*(1+VSD)] or None)."""
+    B, K, V = q_horiz.shape
+    slots = spec_cache_slots(IW, VSD)
+    _check(q_horiz, torch.float32, "q_horiz")
+    _check(cache_rows, torch.float32, "cache_rows", (B, slots, V))
+    _check(cache_tags, torch.int32, "cache_tags", (B, slots))
+    _check(position, torch.int32, "position", (B,))
+    NQ = K * (1 + VSD)
+    pool_q = torch.empty((B, NQ, V), dtype=torch.float32, device=q_horiz.device)
+    source = torch.empty((B, NQ), dtype=torch.int32, device=q_horiz.device) if with_source else None
+    rc = load_library().hawk_pool_build(_ptr(q_horiz), _ptr(cache_rows), _ptr(cache_tags), _ptr(position),
+                                        _ptr(pool_q), _ptr(source), B, K, int(IW), int(VSD), V, _stream())
+    if rc != 0:
+        raise HawkError(rc, "hawk_pool_build")
+    return pool_q, source
+
+
+def pool_sample_workspace_bytes(B: int, NQ: int) -> int:
+    return int(load_library().hawk_pool_sample_workspace_bytes(int(B), int(NQ)))
+
+
+def pool_sample(pool_q: torch.Tensor, u: torch.Tensor, node_q: torch.Tensor, v_begin: int, v_end: int,
+                dev_status: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """One draw per pool row, handed to the tree nodes: returns node_token [B,N] int32."""
+    B, NQ, V = pool_q.shape
+    N = node_q.shape[0]
+    _check(pool_q, torch.float32, "pool_q")
+    _check(u, torch.float32, "u", (B, NQ))
+    _check(node_q, torch.int32, "node_q", (N,))
+    node_token = torch.empty((B, N), dtype=torch.int32, device=pool_q.device)
+    need = pool_sample_workspace_bytes(B, NQ)
+    workspace = torch.empty(max(need, 16), dtype=torch.uint8, device=pool_q.device)
+    rc = load_library().hawk_pool_sample(_ptr(pool_q), _ptr(u), _ptr(node_q), _ptr(node_token), B, NQ, N, V,
+                                         int(v_begin), int(v_end), _ptr(workspace), workspace.numel(),
+                                         _ptr(dev_status), _stream())
+    if rc != 0:
+        raise HawkError(rc, "hawk_pool_sample")
+    return node_token
 
 
 def verify_step_host(args: StepHostArgs) -> None:

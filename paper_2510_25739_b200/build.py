@@ -14,7 +14,7 @@ from pathlib import Path
 PKG = Path(__file__).resolve().parent
 CSRC = PKG / "csrc"
 LIB = PKG / "libhawk_verify.so"
-SOURCES = ["hawk_api.cu", "hawk_accept.cu", "hawk_attn.cu", "hawk_head.cu", "hawk_step.cu"]
+SOURCES = ["hawk_api.cu", "hawk_accept.cu", "hawk_attn.cu", "hawk_head.cu", "hawk_step.cu", "hawk_pool.cu"]
 ARCH_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a"]
 
 

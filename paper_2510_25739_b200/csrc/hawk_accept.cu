@@ -751,6 +751,57 @@ __global__ void __launch_bounds__(NT) tree_rows_kernel(const TreeParams P)
     if (tid == 0) P.verdict[b * P.N + node] = tok >= 0 ? -(P.v_begin + tok) - 2 : -1;
 }
 
+// ------------------------------------------------------------------------------------------------
+// Drawing the candidates (Sec. 4.2: the candidates of the tree are samples from the distributions of
+// the spatial sampling pool): one block per (sequence, pool row) draws one token by inverse CDF in
+// ascending id, with the same scan and search as the correction token above.
+template <int NT, int VPT>
+__global__ void __launch_bounds__(NT) pool_sample_kernel(const float *pool_q, const float *u, int32_t *row_token,
+                                                         int V, int v_begin, int n, int vec_ok)
+{
+    __shared__ RowShared<NT, VPT> sh;
+    const int tid = threadIdx.x;
+    hawk::allow_dependent_launch();
+    hawk::grid_dependency_wait();
+    const float *qrow = pool_q + static_cast<size_t>(blockIdx.x) * V + v_begin;
+    const float ur = u[blockIdx.x];
+    float x[VPT][4], sj[VPT], incl[VPT];
+#pragma unroll
+    for (int j = 0; j < VPT; ++j) {
+        const int e0 = 4 * (j * NT + tid);
+        const float4 q4 = e0 < n ? load4(qrow, e0, n, vec_ok != 0, 0.f) : make_float4(0.f, 0.f, 0.f, 0.f);
+        x[j][0] = fmaxf(q4.x, 0.f);  // (a NaN weight counts as none)
+        x[j][1] = fmaxf(q4.y, 0.f);
+        x[j][2] = fmaxf(q4.z, 0.f);
+        x[j][3] = fmaxf(q4.w, 0.f);
+    }
+    const float total = row_mass<NT, VPT>(x, sj, incl, sh);
+    int tok = -1;
+    if (total > 0.f) tok = row_search<NT, VPT>(x, sj, incl, ur * total, sh);
+    if (tid == 0) row_token[blockIdx.x] = tok >= 0 ? v_begin + tok : -1;
+}
+
+// node_token[b][node] = the draw of the pool row the node's candidate comes from (node 0, the root, gets 0).
+__global__ void pool_scatter_kernel(const int32_t *row_token, const int32_t *node_q, int32_t *node_token, int B, int NQ,
+                                    int N, int32_t *dev_status)
+{
+    hawk::allow_dependent_launch();
+    hawk::grid_dependency_wait();
+    const int idx = blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx >= B * N) return;
+    const int b = idx / N, node = idx - b * N;
+    int tok = 0;
+    if (node > 0) {
+        int r = node_q[node];
+        if (r < 0 || r >= NQ) {
+            if (dev_status) atomicOr(dev_status, HAWK_DEV_BAD_TREE);
+            r = max(0, min(r, NQ - 1));
+        }
+        tok = row_token[b * NQ + r];
+    }
+    node_token[idx] = tok;
+}
+
 // One thread per sequence: follows the verdicts from the root.
 __global__ void tree_walk_kernel(const int32_t *verdict, int B, int N, int max_depth, int32_t *accept_len,
                                  int32_t *out_token, int32_t *path, int32_t *dev_status)
@@ -949,6 +1000,52 @@ extern "C" hawk_status hawk_tree_accept(const float *logits, const float *q_prob
     err = hawk_host::launch_dependent(tree_walk_kernel, dim3((B + 127) / 128), dim3(128), 0, st,
                                       static_cast<const int32_t *>(P.verdict), B, N, path ? max_depth : 0, accept_len,
                                       out_token, path, dev_status);
+    return err == cudaSuccess ? HAWK_OK : HAWK_ERR_CUDA;
+}
+
+
+extern "C" size_t hawk_pool_sample_workspace_bytes(int B, int NQ)
+{
+    if (B <= 0 || NQ <= 0) return 0;
+    return static_cast<size_t>(B) * static_cast<size_t>(NQ) * sizeof(int32_t);
+}
+
+extern "C" hawk_status hawk_pool_sample(const float *pool_q, const float *u, const int32_t *node_q,
+                                        int32_t *node_token, int B, int NQ, int N, int V, int v_begin, int v_end,
+                                        void *workspace, size_t workspace_bytes, int32_t *dev_status,
+                                        hawk_stream_t stream)
+{
+    if (B < 0 || NQ < 0 || N < 0 || V < 0) return HAWK_ERR_SHAPE;
+    if (B == 0) return HAWK_OK;
+    if (!pool_q || !u || !node_q || !node_token) return HAWK_ERR_NULL;
+    if (NQ < 1 || N < 1 || v_begin < 0 || v_end > V || v_begin >= v_end) return HAWK_ERR_SHAPE;
+    const int n = v_end - v_begin;
+    if (n > 32768) return HAWK_ERR_UNSUPPORTED;
+    if (!hawk_host::aligned16(pool_q)) return HAWK_ERR_ALIGN;
+    const size_t need = hawk_pool_sample_workspace_bytes(B, NQ);
+    if (!workspace || workspace_bytes < need) return HAWK_ERR_WORKSPACE;
+    if (!hawk_host::aligned16(workspace)) return HAWK_ERR_ALIGN;
+    if (!hawk_host::is_sm100(nullptr)) return HAWK_ERR_UNSUPPORTED;
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    int32_t *row_token = static_cast<int32_t *>(workspace);
+    const int vec_ok = (V % 4 == 0 && v_begin % 4 == 0) ? 1 : 0;
+    const int grid = B * NQ;
+    cudaError_t err;
+    if (n <= 4096)
+        err = hawk_host::launch_dependent(pool_sample_kernel<256, 4>, dim3(grid), dim3(256), 0, st, pool_q, u, row_token, V,
+                                          v_begin, n, vec_ok);
+    else if (n <= 8192)
+        err = hawk_host::launch_dependent(pool_sample_kernel<512, 4>, dim3(grid), dim3(512), 0, st, pool_q, u, row_token, V,
+                                          v_begin, n, vec_ok);
+    else if (n <= 16384)
+        err = hawk_host::launch_dependent(pool_sample_kernel<1024, 4>, dim3(grid), dim3(1024), 0, st, pool_q, u, row_token,
+                                          V, v_begin, n, vec_ok);
+    else
+        err = hawk_host::launch_dependent(pool_sample_kernel<1024, 8>, dim3(grid), dim3(1024), 0, st, pool_q, u, row_token,
+                                          V, v_begin, n, vec_ok);
+    if (err != cudaSuccess) return HAWK_ERR_CUDA;
+    err = hawk_host::launch_dependent(pool_scatter_kernel, dim3((B * N + 255) / 256), dim3(256), 0, st,
+                                      static_cast<const int32_t *>(row_token), node_q, node_token, B, NQ, N, dev_status);
     return err == cudaSuccess ? HAWK_OK : HAWK_ERR_CUDA;
 }
 

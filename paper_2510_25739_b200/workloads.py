@@ -288,3 +288,24 @@ def draw_tree_uniforms(B: int, N: int, seed: int) -> dict:
     one_below = np.nextafter(np.float32(1.0), np.float32(0.0))
     return dict(u_accept=np.minimum(rng.random((B, N), dtype=np.float32), one_below),
                 u_resample=np.minimum(rng.random((B, N), dtype=np.float32), one_below))
+
+
+# ------------------------------------------------------------------------------------------
+# draft-head outputs for the speculation cache and the sampling pool (Sec. 4.2): random rows only
+# ------------------------------------------------------------------------------------------
+def make_head_probs(B: int, R: int, V: int, v_begin: int, v_end: int, seed: int, sharp: float = 4.0) -> np.ndarray:
+    """[B, R, V] fp32 distributions over the valid ids, normalised exp of sharp * N(0,1): a few ids carry
+    most of the mass, as a trained draft head's output does."""
+    rng = np.random.default_rng(seed + 11)
+    z = sharp * rng.standard_normal((B, R, V))
+    ids = np.arange(V)
+    z = np.where((ids >= v_begin) & (ids < v_end), z, -np.inf)
+    e = np.exp(z - z.max(axis=-1, keepdims=True))
+    return (e / e.sum(axis=-1, keepdims=True)).astype(np.float32)
+
+
+def draw_pool_uniforms(B: int, NQ: int, seed: int) -> np.ndarray:
+    """u [B, NQ] fp32 in [0, 1): one uniform per pool distribution."""
+    rng = np.random.default_rng(seed + 12)
+    u = rng.random((B, NQ), dtype=np.float32)
+    return np.minimum(u, np.nextafter(np.float32(1.0), np.float32(0.0)))
