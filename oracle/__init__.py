@@ -99,6 +99,19 @@ def head_proj(x, w, v_begin=0, v_end=None, fill=np.nan) -> np.ndarray:
     return logits
 
 
+def head_proj_cfg(x, w, cfg_scale, temperature, v_begin=0, v_end=None, fill=np.nan) -> np.ndarray:
+    """x [2B,rows,hidden], w [V,hidden] (uint16 bf16 bits) -> guided logits fp32 [B,rows,V]."""
+    x = _c(x, np.uint16); w = _c(w, np.uint16)
+    S, rows, hidden = x.shape
+    assert S % 2 == 0
+    B, V = S // 2, w.shape[0]
+    v_end = V if v_end is None else v_end
+    guided = np.full((B, rows, V), fill, dtype=np.float32)
+    _load().hawk_oracle_head_proj_cfg(_p(x), _p(w), _p(guided), B, rows, hidden, V, v_begin, v_end,
+                                      ctypes.c_float(cfg_scale), ctypes.c_float(temperature))
+    return guided
+
+
 def target_probs(lc, lu, v_begin, v_end, cfg_scale, temperature, top_k):
     """One position: fp32 rows lc, lu [V] -> (p fp64 [V], flags)."""
     lc = _c(lc, np.float32); lu = _c(lu, np.float32)

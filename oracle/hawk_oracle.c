@@ -511,3 +511,35 @@ void hawk_oracle_pool_sample(const float *pool_q, const float *u, int R, int V, 
         free(w);
     }
 }
+
+/* ------------------------------------------------------------------------------------------
+ * Steps 2 and 3a's first half in one: the output head followed by the guidance combine and the
+ * temperature (generation settings of Sec. 5), for callers that never need the two logit rows:
+ *   guided[b*rows + i][v] = (lu + s*(lc - lu)) / T,  lc / lu the head's logits (rounded to fp32 as
+ *   hawk_oracle_head_proj returns them) of rows (b, i) and (B + b, i) of x,
+ * evaluated in fp32 as subtract, fused multiply-add, divide like hawk_oracle_target_probs.
+ *   x bf16 [2B][rows][hidden], w bf16 [V][hidden], guided fp32 [B][rows][V]
+ * ------------------------------------------------------------------------------------------ */
+void hawk_oracle_head_proj_cfg(const uint16_t *x, const uint16_t *w, float *guided, int B, int rows,
+                               int hidden, int V, int v_begin, int v_end, float cfg_scale,
+                               float temperature)
+{
+    int pairs = B * rows;
+#pragma omp parallel for schedule(static)
+    for (int m = 0; m < pairs; ++m) {
+        const uint16_t *xc = x + (size_t)m * hidden, *xu = x + (size_t)(pairs + m) * hidden;
+        for (int v = v_begin; v < v_end; ++v) {
+            const uint16_t *wr = w + (size_t)v * hidden;
+            double acc_c = 0.0, acc_u = 0.0;
+            for (int c = 0; c < hidden; ++c) {
+                acc_c += bf16_to_double(xc[c]) * bf16_to_double(wr[c]);
+                acc_u += bf16_to_double(xu[c]) * bf16_to_double(wr[c]);
+            }
+            float lc = (float)acc_c, lu = (float)acc_u;
+            volatile float diff = lc - lu;
+            volatile float g = fmaf(cfg_scale, diff, lu);
+            volatile float scaled = g / temperature;
+            guided[(size_t)m * V + v] = scaled;
+        }
+    }
+}
