@@ -227,6 +227,16 @@ def run_accept(cfg, r, hawk):
                     out_token=r.out_token, workspace=r.acc_ws, dev_status=r.status)
 
 
+def run_head_cfg(cfg, r, hawk):
+    hawk.head_proj_cfg(r.x.view(cfg.S, cfg.K, cfg.hidden), r.w, cfg.cfg_scale, cfg.temperature, cfg.v_begin, cfg.v_end,
+                       guided=r.guided, dev_status=r.status)
+
+
+def run_accept_guided(cfg, r, hawk):
+    hawk.cfg_accept_guided(r.guided, r.q_probs, r.draft, r.u_accept, r.u_resample, cfg.v_begin, cfg.v_end, cfg.top_k,
+                           accept_len=r.accept_len2, out_token=r.out_token2, workspace=r.acc_ws, dev_status=r.status)
+
+
 def make_event(torch):
     try:
         return torch.cuda.Event(enable_timing=True, external=True), True
@@ -435,6 +445,51 @@ def main():
             a1.record(stream)
             stream.synchronize()
             kernels[name] = a0.elapsed_time(a1) * 1e3 / (n * n_rep)   # us per launch
+    # ---- the two-call form: guidance combined in the head's epilogue, accept reads one guided row per position
+    for r in reps:
+        r.guided = torch.zeros((cfg.B, cfg.K, cfg.V), dtype=torch.float32, device="cuda")
+        r.accept_len2 = torch.empty_like(r.accept_len)
+        r.out_token2 = torch.empty_like(r.out_token)
+    with torch.cuda.stream(stream):
+        for r in reps:
+            run_head_cfg(cfg, r, hawk); run_accept_guided(cfg, r, hawk)
+        stream.synchronize()
+        for name, fn in (("head_cfg", run_head_cfg), ("accept_guided", run_accept_guided)):
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=stream):
+                for r in reps:
+                    fn(cfg, r, hawk)
+            for _ in range(3):
+                g.replay()
+            stream.synchronize()
+            a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            n = max(3, min(200, K_steps // n_rep + 1))
+            a0.record(stream)
+            for _ in range(n):
+                g.replay()
+            a1.record(stream)
+            stream.synchronize()
+            kernels[name] = a0.elapsed_time(a1) * 1e3 / (n * n_rep)
+        graphs2 = []
+        for r in reps:
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=stream):
+                run_attn(cfg, r, hawk)
+                run_head_cfg(cfg, r, hawk)
+                run_accept_guided(cfg, r, hawk)
+            graphs2.append(g)
+        for i in range(W):
+            graphs2[i % n_rep].replay()
+        stream.synchronize()
+        a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a0.record(stream)
+        for i in range(K_steps):
+            graphs2[i % n_rep].replay()
+        a1.record(stream)
+        stream.synchronize()
+        us_step2 = a0.elapsed_time(a1) * 1e3 / K_steps
+    same = all(bool(torch.equal(r.accept_len, r.accept_len2)) and bool(torch.equal(r.out_token, r.out_token2))
+               for r in reps)
     rej = sum(int((r.accept_len < cfg.K).sum().item()) for r in reps) / n_rep
     mean_len = float(sum(float(r.accept_len.float().mean().item()) for r in reps) / n_rep)
     q_rows = sum(int(r.accept_len.clamp(max=cfg.K - 1).add(1).sum().item()) for r in reps) / n_rep
@@ -449,6 +504,11 @@ def main():
                    "frac_hbm": accept_bytes(cfg, cfg.B * cfg.K) / kernels["accept"] / 1e3 / peaks["hbm_gbs"],
                    "bytes_counted": "both logit rows of every position + one q row per position"},
         "mean_accept_len": mean_len, "sequences_with_rejection": rej, "q_rows_on_chain": q_rows,
+        "two_call_form": {
+            "what": "hawk_head_proj_cfg + hawk_cfg_accept_guided: one guided logits row per position crosses HBM",
+            "head_cfg_us": kernels["head_cfg"], "accept_guided_us": kernels["accept_guided"],
+            "step_us": us_step2, "positions_per_s": positions * world / (us_step2 * 1e-6),
+            "same_verdicts_as_three_calls": same},
     }
 
     # ---- candidate-tree verification (not part of the timed step): a (3, 2, 2) tree, 22 nodes per sequence

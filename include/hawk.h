@@ -10,7 +10,8 @@
  *   hawk_cfg_accept   guidance combine, temperature, top-k, softmax and speculative rejection
  *                     sampling, returning the accepted length and the correction token;
  *   hawk_tree_accept  the same for a candidate tree with several candidates per depth.
- *   hawk_spec_cache_*, hawk_pool_*  the cache of vertical predictions and the sampling pool that feed it.
+ *   hawk_spec_cache_*, hawk_pool_*  the cache of vertical predictions and the sampling pool that feed it;
+ *   hawk_head_proj_cfg, hawk_*_accept_guided  the head with the guidance combine in its epilogue.
  *
  * Conventions common to all entry points
  *   - Every pointer is a DEVICE pointer owned by the caller unless the comment says "host".  The
@@ -220,6 +221,44 @@ hawk_status hawk_tree_accept(const float *logits, const float *q_probs, const in
                              float cfg_scale, float temperature, int top_k, int max_depth,
                              int32_t *accept_len, int32_t *out_token, int32_t *path, void *workspace,
                              size_t workspace_bytes, int32_t *dev_status, hawk_stream_t stream);
+
+/* ------------------------------------------------------------------------------------------------
+ * Guidance fused into the output head (generation settings of Sec. 5: guidance scale and temperature
+ * applied to the target's logits before top-k and sampling).  The paper does not separate these
+ * steps; the three calls below are the two-call form of hawk_head_proj + hawk_cfg_accept /
+ * hawk_tree_accept in which the conditional and the unconditional logit rows never reach memory.
+ *
+ * hawk_head_proj_cfg: guided[b*rows + i][v] = (lu + cfg_scale * (lc - lu)) / temperature, with
+ *     lc = sum_c x[b*rows + i][c] * w[v][c],   lu = sum_c x[(B + b)*rows + i][c] * w[v][c]
+ * for v_begin <= v < v_end: the accumulators of hawk_head_proj combined in fp32 by subtract, fused
+ * multiply-add, divide (step 1 of hawk_cfg_accept, on the same numbers), so the two-call form decides
+ * exactly as the three-call form does.
+ *   x       bf16 [2B][rows][hidden]   conditional streams first, as everywhere
+ *   w       bf16 [V][hidden]
+ *   guided  fp32 [B][rows][V]         columns outside [v_begin, v_end) are not written
+ * Supported: hidden a multiple of 64.  Errors as hawk_head_proj, plus PARAM (temperature <= 0, NaN, inf).
+ *
+ * hawk_cfg_accept_guided / hawk_tree_accept_guided: hawk_cfg_accept / hawk_tree_accept from step 2 on,
+ * reading `guided` fp32 [B][K(+1)][V] / [B][N][V] instead of the two logit rows (no guidance scale,
+ * no temperature: both are already applied).  NaN or +inf in `guided` is treated as -inf and flagged
+ * HAWK_DEV_NONFINITE.  All other arguments, limits, workspaces and errors as the calls they mirror.
+ * ---------------------------------------------------------------------------------------------- */
+hawk_status hawk_head_proj_cfg(const void *x, const void *w, float *guided, int B, int rows, int hidden, int V,
+                               int v_begin, int v_end, float cfg_scale, float temperature, int32_t *dev_status,
+                               hawk_stream_t stream);
+
+hawk_status hawk_cfg_accept_guided(const float *guided, const float *q_probs, const int32_t *draft,
+                                   const float *u_accept, const float *u_resample, int B, int K, int V, int v_begin,
+                                   int v_end, int top_k, int has_bonus_row, int32_t *accept_len, int32_t *out_token,
+                                   float *p_debug, void *workspace, size_t workspace_bytes, int32_t *dev_status,
+                                   hawk_stream_t stream);
+
+hawk_status hawk_tree_accept_guided(const float *guided, const float *q_probs, const int32_t *node_token,
+                                    const int32_t *node_q, const int32_t *child_begin, const float *u_accept,
+                                    const float *u_resample, int B, int N, int NQ, int V, int v_begin, int v_end,
+                                    int top_k, int max_depth, int32_t *accept_len, int32_t *out_token, int32_t *path,
+                                    void *workspace, size_t workspace_bytes, int32_t *dev_status,
+                                    hawk_stream_t stream);
 
 /* ------------------------------------------------------------------------------------------------
  * Speculation cache and spatial sampling pool (Sec. 4.2, "Dual Direction Drafting Heads" and "Spatial

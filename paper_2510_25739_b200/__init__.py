@@ -15,6 +15,7 @@ _BINDING_NAMES = (
     "cfg_accept_noalloc", "cfg_accept_noalloc_max_rows", "tree_accept", "verify_attn_tree",
     "spec_cache_slots", "spec_cache_slot", "spec_cache_new", "spec_cache_clear", "spec_cache_put",
     "pool_build", "pool_sample", "pool_sample_workspace_bytes",
+    "head_proj_cfg", "cfg_accept_guided", "tree_accept_guided",
 )
 
 

@@ -28,6 +28,7 @@ EXPORTS = (
     "hawk_tree_accept_workspace_bytes", "hawk_tree_accept", "hawk_verify_attn_tree",
     "hawk_spec_cache_slots", "hawk_spec_cache_slot", "hawk_spec_cache_clear", "hawk_spec_cache_put",
     "hawk_pool_build", "hawk_pool_sample_workspace_bytes", "hawk_pool_sample",
+    "hawk_head_proj_cfg", "hawk_cfg_accept_guided", "hawk_tree_accept_guided",
 )
 
 
@@ -96,6 +97,12 @@ def load_library() -> ctypes.CDLL:
     lib.hawk_tree_accept_workspace_bytes.argtypes = [i32, i32]
     lib.hawk_tree_accept.restype = i32
     lib.hawk_tree_accept.argtypes = [vp] * 7 + [i32] * 6 + [f32, f32, i32, i32] + [vp, vp, vp, vp, sz, vp, vp]
+    lib.hawk_head_proj_cfg.restype = i32
+    lib.hawk_head_proj_cfg.argtypes = [vp, vp, vp, i32, i32, i32, i32, i32, i32, f32, f32, vp, vp]
+    lib.hawk_cfg_accept_guided.restype = i32
+    lib.hawk_cfg_accept_guided.argtypes = [vp] * 5 + [i32] * 7 + [vp, vp, vp, vp, sz, vp, vp]
+    lib.hawk_tree_accept_guided.restype = i32
+    lib.hawk_tree_accept_guided.argtypes = [vp] * 7 + [i32] * 8 + [vp, vp, vp, vp, sz, vp, vp]
     lib.hawk_spec_cache_slots.restype = i32
     lib.hawk_spec_cache_slots.argtypes = [i32, i32]
     lib.hawk_spec_cache_slot.restype = i32
@@ -208,6 +215,65 @@ def head_proj(x: torch.Tensor, w: torch.Tensor, v_begin: int = 0, v_end: Optiona
     return logits
 
 
+def head_proj_cfg(x: torch.Tensor, w: torch.Tensor, cfg_scale: float, temperature: float, v_begin: int = 0,
+                  v_end: Optional[int] = None, guided: Optional[torch.Tensor] = None,
+                  dev_status: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """x [2B,rows,hidden], w [V,hidden] (bf16) -> guided logits [B,rows,V] fp32 (columns [v_begin,v_end) written)."""
+    lib = load_library()
+    S, rows, hidden = x.shape
+    if S % 2:
+        raise ValueError("x: the first dimension holds B conditional then B unconditional streams")
+    B = S // 2
+    V = w.shape[0]
+    v_end = V if v_end is None else v_end
+    _check(x, torch.bfloat16, "x")
+    _check(w, torch.bfloat16, "w", (V, hidden))
+    if guided is None:
+        guided = torch.empty((B, rows, V), dtype=torch.float32, device=x.device)
+    _check(guided, torch.float32, "guided", (B, rows, V))
+    rc = lib.hawk_head_proj_cfg(_ptr(x), _ptr(w), _ptr(guided), B, rows, hidden, V, int(v_begin), int(v_end),
+                                float(cfg_scale), float(temperature), _ptr(dev_status), _stream())
+    if rc != 0:
+        raise HawkError(rc, "hawk_head_proj_cfg")
+    return guided
+
+
+def cfg_accept_guided(guided: torch.Tensor, q_probs: torch.Tensor, draft: torch.Tensor, u_accept: torch.Tensor,
+                      u_resample: torch.Tensor, v_begin: int, v_end: int, top_k: int, has_bonus_row: bool = False,
+                      accept_len: Optional[torch.Tensor] = None, out_token: Optional[torch.Tensor] = None,
+                      p_debug: Optional[torch.Tensor] = None, workspace: Optional[torch.Tensor] = None,
+                      dev_status: Optional[torch.Tensor] = None):
+    """guided [B,K(+1),V] fp32 (from head_proj_cfg), otherwise as cfg_accept -> (accept_len, out_token)."""
+    lib = load_library()
+    B, K, V = q_probs.shape
+    rows = K + (1 if has_bonus_row else 0)
+    _check(guided, torch.float32, "guided", (B, rows, V))
+    _check(q_probs, torch.float32, "q_probs")
+    _check(draft, torch.int32, "draft", (B, K))
+    _check(u_accept, torch.float32, "u_accept", (B, K))
+    _check(u_resample, torch.float32, "u_resample", (B, K + 1))
+    dev = guided.device
+    if accept_len is None:
+        accept_len = torch.empty(B, dtype=torch.int32, device=dev)
+    if out_token is None:
+        out_token = torch.empty(B, dtype=torch.int32, device=dev)
+    _check(accept_len, torch.int32, "accept_len", (B,))
+    _check(out_token, torch.int32, "out_token", (B,))
+    if p_debug is not None:
+        _check(p_debug, torch.float32, "p_debug", (B, rows, V))
+    need = cfg_accept_workspace_bytes(B, K, V)
+    if workspace is None:
+        workspace = torch.empty(max(need, 16), dtype=torch.uint8, device=dev)
+    ws_bytes = workspace.numel() * workspace.element_size()
+    rc = lib.hawk_cfg_accept_guided(_ptr(guided), _ptr(q_probs), _ptr(draft), _ptr(u_accept), _ptr(u_resample), B, K, V,
+                                    int(v_begin), int(v_end), int(top_k), int(bool(has_bonus_row)), _ptr(accept_len),
+                                    _ptr(out_token), _ptr(p_debug), _ptr(workspace), ws_bytes, _ptr(dev_status),
+                                    _stream())
+    if rc != 0:
+        raise HawkError(rc, "hawk_cfg_accept_guided")
+    return accept_len, out_token
+
+
 def cfg_accept_workspace_bytes(B: int, K: int, V: int) -> int:
     return int(load_library().hawk_cfg_accept_workspace_bytes(B, K, V))
 
@@ -308,6 +374,37 @@ def tree_accept(logits: torch.Tensor, q_probs: torch.Tensor, node_token: torch.T
                               _stream())
     if rc != 0:
         raise HawkError(rc, "hawk_tree_accept")
+    return accept_len, out_token, path
+
+
+def tree_accept_guided(guided: torch.Tensor, q_probs: torch.Tensor, node_token: torch.Tensor, node_q: torch.Tensor,
+                       child_begin: torch.Tensor, u_accept: torch.Tensor, u_resample: torch.Tensor, v_begin: int,
+                       v_end: int, top_k: int, max_depth: Optional[int] = None,
+                       dev_status: Optional[torch.Tensor] = None):
+    """guided [B,N,V] fp32 (from head_proj_cfg), otherwise as tree_accept -> (accept_len, out_token, path)."""
+    lib = load_library()
+    B, NQ, V = q_probs.shape
+    N = node_q.shape[0]
+    max_depth = N if max_depth is None else int(max_depth)
+    _check(guided, torch.float32, "guided", (B, N, V))
+    _check(q_probs, torch.float32, "q_probs")
+    _check(node_token, torch.int32, "node_token", (B, N))
+    _check(node_q, torch.int32, "node_q", (N,))
+    _check(child_begin, torch.int32, "child_begin", (N + 1,))
+    _check(u_accept, torch.float32, "u_accept", (B, N))
+    _check(u_resample, torch.float32, "u_resample", (B, N))
+    dev = guided.device
+    accept_len = torch.empty(B, dtype=torch.int32, device=dev)
+    out_token = torch.empty(B, dtype=torch.int32, device=dev)
+    path = torch.empty((B, max_depth), dtype=torch.int32, device=dev)
+    need = int(lib.hawk_tree_accept_workspace_bytes(B, N))
+    workspace = torch.empty(max(need, 16), dtype=torch.uint8, device=dev)
+    rc = lib.hawk_tree_accept_guided(_ptr(guided), _ptr(q_probs), _ptr(node_token), _ptr(node_q), _ptr(child_begin),
+                                     _ptr(u_accept), _ptr(u_resample), B, N, NQ, V, int(v_begin), int(v_end),
+                                     int(top_k), max_depth, _ptr(accept_len), _ptr(out_token), _ptr(path),
+                                     _ptr(workspace), workspace.numel(), _ptr(dev_status), _stream())
+    if rc != 0:
+        raise HawkError(rc, "hawk_tree_accept_guided")
     return accept_len, out_token, path
 
 

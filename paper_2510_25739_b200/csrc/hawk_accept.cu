@@ -40,6 +40,7 @@ struct AcceptParams {
     float cfg_scale, temperature;
     int top_k;
     int vec_ok;
+    int guided_in;     // logits is [B][rows][V] of guided logits instead of [2B][rows][V]
     int32_t *row_out;  // [B][rows]
     float *p_debug;
     int32_t *dev_status;
@@ -185,7 +186,10 @@ struct RowShared {
 // or +inf, as opposed to a plain -inf mask) is sorted out afterwards, and only by threads that met one.
 // `full` (block-uniform): the row fills the block exactly and is 16-byte aligned, so no id needs a
 // bounds check.
-template <int NT, int VPT>
+// GUIDED: lc already holds guided logits (the head projection combined the two
+// streams); the caller passes temperature 1, so the arithmetic below returns every finite value as it
+// is (fma(s, c - c, c) = c) and the row is read once.
+template <int NT, int VPT, bool GUIDED>
 __device__ __forceinline__ void row_load(const float *lc, const float *lu, int n, bool vec_ok, bool full,
                                          float cfg_scale, float temperature, float (&x)[VPT][4], float &mx,
                                          float &mn, int &cnt, int &flags)
@@ -198,14 +202,14 @@ __device__ __forceinline__ void row_load(const float *lc, const float *lu, int n
 #pragma unroll
         for (int j = 0; j < VPT; ++j) {  // all loads in flight before the first use
             c4[j] = ld_stream4(lc + 4 * (j * NT + tid));
-            u4[j] = ld_stream4(lu + 4 * (j * NT + tid));
+            u4[j] = GUIDED ? c4[j] : ld_stream4(lu + 4 * (j * NT + tid));
         }
     } else {
 #pragma unroll
         for (int j = 0; j < VPT; ++j) {
             const int e0 = 4 * (j * NT + tid);
             c4[j] = e0 < n ? load4(lc, e0, n, vec_ok, -CUDART_INF_F) : make_float4(-CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F);
-            u4[j] = e0 < n ? load4(lu, e0, n, vec_ok, -CUDART_INF_F) : c4[j];
+            u4[j] = (!GUIDED && e0 < n) ? load4(lu, e0, n, vec_ok, -CUDART_INF_F) : c4[j];
         }
     }
     bool odd = false;  // met an id whose inputs or result are not finite
@@ -230,7 +234,7 @@ __device__ __forceinline__ void row_load(const float *lc, const float *lu, int n
         for (int j = 0; j < VPT; ++j) {
             const int e0 = 4 * (j * NT + tid);
             if (e0 >= n) break;
-            const float4 a = load4(lc, e0, n, vec_ok, -CUDART_INF_F), b = load4(lu, e0, n, vec_ok, -CUDART_INF_F);
+            const float4 a = load4(lc, e0, n, vec_ok, -CUDART_INF_F), b = GUIDED ? a : load4(lu, e0, n, vec_ok, -CUDART_INF_F);
             int fl = 0;
             (void)guided(a.x, b.x, cfg_scale, temperature, unit_T, fl);
             (void)guided(a.y, b.y, cfg_scale, temperature, unit_T, fl);
@@ -484,7 +488,7 @@ __device__ __forceinline__ int row_search(const float (&rr)[VPT][4], const float
 
 // Chain verification: one block per (sequence, draft position) row.
 // NT threads, VPT float4 loads per thread: the block holds up to 4 * NT * VPT valid ids of its row.
-template <int NT, int VPT>
+template <int NT, int VPT, bool GUIDED>
 __global__ void __launch_bounds__(NT) accept_rows_kernel(const AcceptParams P)
 {
     __shared__ RowShared<NT, VPT> sh;
@@ -498,7 +502,7 @@ __global__ void __launch_bounds__(NT) accept_rows_kernel(const AcceptParams P)
     const int n = P.n;
     const bool vec_ok = P.vec_ok != 0;
     const float *lc = P.logits + (static_cast<size_t>(b) * P.rows + i) * P.V + P.v_begin;
-    const float *lu = P.logits + (static_cast<size_t>(P.B + b) * P.rows + i) * P.V + P.v_begin;
+    const float *lu = GUIDED ? nullptr : P.logits + (static_cast<size_t>(P.B + b) * P.rows + i) * P.V + P.v_begin;
     const float *qrow = bonus ? nullptr : P.q + (static_cast<size_t>(b) * P.K + i) * P.V + P.v_begin;
     int flags = 0;
 
@@ -510,7 +514,7 @@ __global__ void __launch_bounds__(NT) accept_rows_kernel(const AcceptParams P)
     float x[VPT][4];
     float mx, mn;
     int cnt;
-    row_load<NT, VPT>(lc, lu, n, vec_ok, vec_ok && n == 4 * NT * VPT, P.cfg_scale, P.temperature, x, mx, mn, cnt, flags);
+    row_load<NT, VPT, GUIDED>(lc, lu, n, vec_ok, vec_ok && n == 4 * NT * VPT, P.cfg_scale, P.temperature, x, mx, mn, cnt, flags);
 
     float qx = 0.f;
     if (!bonus) {
@@ -620,11 +624,12 @@ struct TreeParams {
     float cfg_scale, temperature;
     int top_k;
     int vec_ok;
+    int guided_in;     // logits is [B][N][V] of guided logits instead of [2B][N][V]
     int32_t *verdict;  // [B][N]: >= 0 the child that passed; -1 stop without a token; <= -2 stop, token = -v - 2
     int32_t *dev_status;
 };
 
-template <int NT, int VPT>
+template <int NT, int VPT, bool GUIDED>
 __global__ void __launch_bounds__(NT) tree_rows_kernel(const TreeParams P)
 {
     __shared__ RowShared<NT, VPT> sh;
@@ -638,7 +643,7 @@ __global__ void __launch_bounds__(NT) tree_rows_kernel(const TreeParams P)
     const int n = P.n;
     const bool vec_ok = P.vec_ok != 0;
     const float *lc = P.logits + (static_cast<size_t>(b) * P.N + node) * P.V + P.v_begin;
-    const float *lu = P.logits + (static_cast<size_t>(P.B + b) * P.N + node) * P.V + P.v_begin;
+    const float *lu = GUIDED ? nullptr : P.logits + (static_cast<size_t>(P.B + b) * P.N + node) * P.V + P.v_begin;
     int flags = 0;
 
     // children of the node; ids must grow along the walk so that it ends
@@ -667,7 +672,7 @@ __global__ void __launch_bounds__(NT) tree_rows_kernel(const TreeParams P)
     float x[VPT][4];
     float mx, mn;
     int cnt;
-    row_load<NT, VPT>(lc, lu, n, vec_ok, vec_ok && n == 4 * NT * VPT, P.cfg_scale, P.temperature, x, mx, mn, cnt, flags);
+    row_load<NT, VPT, GUIDED>(lc, lu, n, vec_ok, vec_ok && n == 4 * NT * VPT, P.cfg_scale, P.temperature, x, mx, mn, cnt, flags);
 
     if (tid < nc) {
         if (my_tok < P.v_begin || my_tok >= P.v_begin + n) {
@@ -860,13 +865,17 @@ __global__ void accept_finalize_kernel(const int32_t *row_out, int B, int K, int
 template <int NT, int VPT>
 cudaError_t launch_rows(const AcceptParams &P, int grid, cudaStream_t stream)
 {
-    return hawk_host::launch_dependent(accept_rows_kernel<NT, VPT>, dim3(grid), dim3(NT), 0, stream, P);
+    if (P.guided_in)
+        return hawk_host::launch_dependent(accept_rows_kernel<NT, VPT, true>, dim3(grid), dim3(NT), 0, stream, P);
+    return hawk_host::launch_dependent(accept_rows_kernel<NT, VPT, false>, dim3(grid), dim3(NT), 0, stream, P);
 }
 
 template <int NT, int VPT>
 cudaError_t launch_tree_rows(const TreeParams &P, int grid, cudaStream_t stream)
 {
-    return hawk_host::launch_dependent(tree_rows_kernel<NT, VPT>, dim3(grid), dim3(NT), 0, stream, P);
+    if (P.guided_in)
+        return hawk_host::launch_dependent(tree_rows_kernel<NT, VPT, true>, dim3(grid), dim3(NT), 0, stream, P);
+    return hawk_host::launch_dependent(tree_rows_kernel<NT, VPT, false>, dim3(grid), dim3(NT), 0, stream, P);
 }
 
 }  // namespace
@@ -878,12 +887,12 @@ extern "C" size_t hawk_cfg_accept_workspace_bytes(int B, int K, int V)
     return static_cast<size_t>(B) * static_cast<size_t>(K + 1) * sizeof(int32_t);
 }
 
-extern "C" hawk_status hawk_cfg_accept(const float *logits, const float *q_probs, const int32_t *draft,
-                                       const float *u_accept, const float *u_resample, int B, int K, int V,
-                                       int v_begin, int v_end, float cfg_scale, float temperature, int top_k,
-                                       int has_bonus_row, int32_t *accept_len, int32_t *out_token, float *p_debug,
-                                       void *workspace, size_t workspace_bytes, int32_t *dev_status,
-                                       hawk_stream_t stream)
+namespace {
+hawk_status cfg_accept_impl(const float *logits, int guided_in, const float *q_probs, const int32_t *draft,
+                            const float *u_accept, const float *u_resample, int B, int K, int V, int v_begin,
+                            int v_end, float cfg_scale, float temperature, int top_k, int has_bonus_row,
+                            int32_t *accept_len, int32_t *out_token, float *p_debug, void *workspace,
+                            size_t workspace_bytes, int32_t *dev_status, hawk_stream_t stream)
 {
     if (B < 0 || K < 0 || V < 0) return HAWK_ERR_SHAPE;
     if (B == 0) return HAWK_OK;
@@ -918,6 +927,7 @@ extern "C" hawk_status hawk_cfg_accept(const float *logits, const float *q_probs
     P.temperature = temperature;
     P.top_k = top_k;
     P.vec_ok = (V % 4 == 0 && v_begin % 4 == 0) ? 1 : 0;
+    P.guided_in = guided_in;
     P.row_out = static_cast<int32_t *>(workspace);
     P.p_debug = p_debug;
     P.dev_status = dev_status;
@@ -934,6 +944,31 @@ extern "C" hawk_status hawk_cfg_accept(const float *logits, const float *q_probs
                                       static_cast<const int32_t *>(P.row_out), B, K, P.rows, accept_len, out_token);
     return err == cudaSuccess ? HAWK_OK : HAWK_ERR_CUDA;
 }
+}  // namespace
+
+extern "C" hawk_status hawk_cfg_accept(const float *logits, const float *q_probs, const int32_t *draft,
+                                       const float *u_accept, const float *u_resample, int B, int K, int V,
+                                       int v_begin, int v_end, float cfg_scale, float temperature, int top_k,
+                                       int has_bonus_row, int32_t *accept_len, int32_t *out_token, float *p_debug,
+                                       void *workspace, size_t workspace_bytes, int32_t *dev_status,
+                                       hawk_stream_t stream)
+{
+    return cfg_accept_impl(logits, 0, q_probs, draft, u_accept, u_resample, B, K, V, v_begin, v_end, cfg_scale,
+                           temperature, top_k, has_bonus_row, accept_len, out_token, p_debug, workspace,
+                           workspace_bytes, dev_status, stream);
+}
+
+extern "C" hawk_status hawk_cfg_accept_guided(const float *guided, const float *q_probs, const int32_t *draft,
+                                              const float *u_accept, const float *u_resample, int B, int K, int V,
+                                              int v_begin, int v_end, int top_k, int has_bonus_row,
+                                              int32_t *accept_len, int32_t *out_token, float *p_debug,
+                                              void *workspace, size_t workspace_bytes, int32_t *dev_status,
+                                              hawk_stream_t stream)
+{
+    return cfg_accept_impl(guided, 1, q_probs, draft, u_accept, u_resample, B, K, V, v_begin, v_end, 1.0f, 1.0f, top_k,
+                           has_bonus_row, accept_len, out_token, p_debug, workspace, workspace_bytes, dev_status,
+                           stream);
+}
 
 
 extern "C" size_t hawk_tree_accept_workspace_bytes(int B, int N)
@@ -942,12 +977,13 @@ extern "C" size_t hawk_tree_accept_workspace_bytes(int B, int N)
     return static_cast<size_t>(B) * static_cast<size_t>(N) * sizeof(int32_t);
 }
 
-extern "C" hawk_status hawk_tree_accept(const float *logits, const float *q_probs, const int32_t *node_token,
-                                        const int32_t *node_q, const int32_t *child_begin, const float *u_accept,
-                                        const float *u_resample, int B, int N, int NQ, int V, int v_begin,
-                                        int v_end, float cfg_scale, float temperature, int top_k, int max_depth,
-                                        int32_t *accept_len, int32_t *out_token, int32_t *path, void *workspace,
-                                        size_t workspace_bytes, int32_t *dev_status, hawk_stream_t stream)
+namespace {
+hawk_status tree_accept_impl(const float *logits, int guided_in, const float *q_probs, const int32_t *node_token,
+                             const int32_t *node_q, const int32_t *child_begin, const float *u_accept,
+                             const float *u_resample, int B, int N, int NQ, int V, int v_begin, int v_end,
+                             float cfg_scale, float temperature, int top_k, int max_depth, int32_t *accept_len,
+                             int32_t *out_token, int32_t *path, void *workspace, size_t workspace_bytes,
+                             int32_t *dev_status, hawk_stream_t stream)
 {
     if (B < 0 || N < 0 || NQ < 0 || V < 0 || max_depth < 0) return HAWK_ERR_SHAPE;
     if (B == 0) return HAWK_OK;
@@ -986,6 +1022,7 @@ extern "C" hawk_status hawk_tree_accept(const float *logits, const float *q_prob
     P.temperature = temperature;
     P.top_k = top_k;
     P.vec_ok = (V % 4 == 0 && v_begin % 4 == 0) ? 1 : 0;
+    P.guided_in = guided_in;
     P.verdict = static_cast<int32_t *>(workspace);
     P.dev_status = dev_status;
 
@@ -1001,6 +1038,32 @@ extern "C" hawk_status hawk_tree_accept(const float *logits, const float *q_prob
                                       static_cast<const int32_t *>(P.verdict), B, N, path ? max_depth : 0, accept_len,
                                       out_token, path, dev_status);
     return err == cudaSuccess ? HAWK_OK : HAWK_ERR_CUDA;
+}
+}  // namespace
+
+extern "C" hawk_status hawk_tree_accept(const float *logits, const float *q_probs, const int32_t *node_token,
+                                        const int32_t *node_q, const int32_t *child_begin, const float *u_accept,
+                                        const float *u_resample, int B, int N, int NQ, int V, int v_begin,
+                                        int v_end, float cfg_scale, float temperature, int top_k, int max_depth,
+                                        int32_t *accept_len, int32_t *out_token, int32_t *path, void *workspace,
+                                        size_t workspace_bytes, int32_t *dev_status, hawk_stream_t stream)
+{
+    return tree_accept_impl(logits, 0, q_probs, node_token, node_q, child_begin, u_accept, u_resample, B, N, NQ, V,
+                            v_begin, v_end, cfg_scale, temperature, top_k, max_depth, accept_len, out_token, path,
+                            workspace, workspace_bytes, dev_status, stream);
+}
+
+extern "C" hawk_status hawk_tree_accept_guided(const float *guided, const float *q_probs, const int32_t *node_token,
+                                               const int32_t *node_q, const int32_t *child_begin,
+                                               const float *u_accept, const float *u_resample, int B, int N, int NQ,
+                                               int V, int v_begin, int v_end, int top_k, int max_depth,
+                                               int32_t *accept_len, int32_t *out_token, int32_t *path,
+                                               void *workspace, size_t workspace_bytes, int32_t *dev_status,
+                                               hawk_stream_t stream)
+{
+    return tree_accept_impl(guided, 1, q_probs, node_token, node_q, child_begin, u_accept, u_resample, B, N, NQ, V,
+                            v_begin, v_end, 1.0f, 1.0f, top_k, max_depth, accept_len, out_token, path, workspace,
+                            workspace_bytes, dev_status, stream);
 }
 
 

@@ -11,6 +11,13 @@
 //   warps 2..5  epilogue: tcgen05.ld of the fp32 accumulator (lane = token id, column = token row),
 //               coalesced 128-byte stores into logits[token][vocab]
 // The accumulator is double-buffered in TMEM so the epilogue of one tile overlaps the MMAs of the next.
+//
+// hawk_head_proj_cfg runs the same kernel with the two guidance streams of a position side by side in
+// one tile: columns [0, BN/2) hold conditional token rows, columns [BN/2, BN) the unconditional rows of
+// the same (sequence, position) pairs (two X boxes per stage).  The epilogue combines the two
+// accumulators of a pair (subtract, fused multiply-add, divide: the arithmetic of the accept kernels)
+// and writes ONE row of guided logits, so the logits cross HBM half as often on the way out and half
+// as often on the way into the accept stage.
 #include "hawk_common.cuh"
 
 namespace {
@@ -32,6 +39,8 @@ struct HeadParams {
     int tiles_n;   // token tiles
     int stages;
     int stage_bytes;
+    int pairs;     // 0: plain logits; > 0: guided logits of this many (sequence, position) pairs
+    float cfg_scale, temperature;
     int32_t *dev_status;
 };
 
@@ -94,7 +103,14 @@ __global__ void __launch_bounds__(kHeadThreads, 1) head_proj_kernel(const __grid
                     uint8_t *a = smem + static_cast<size_t>(st) * P.stage_bytes;
                     mbar_arrive_expect_tx(&full_bar[st], tx_bytes);
                     tma_load_2d(a, &map_w, kb * kBK, row_w, &full_bar[st]);
-                    tma_load_2d(a + kATileBytes, &map_x, kb * kBK, row_x, &full_bar[st]);
+                    if (P.pairs == 0) {
+                        tma_load_2d(a + kATileBytes, &map_x, kb * kBK, row_x, &full_bar[st]);
+                    } else {  // conditional rows of the tile's pairs, then their unconditional rows
+                        const int half = P.BN / 2;
+                        tma_load_2d(a + kATileBytes, &map_x, kb * kBK, tn * half, &full_bar[st]);
+                        tma_load_2d(a + kATileBytes + half * kBK * 2, &map_x, kb * kBK, P.pairs + tn * half,
+                                    &full_bar[st]);
+                    }
                     ++issued;
                     if (++st == P.stages) {
                         st = 0;
@@ -165,15 +181,36 @@ __global__ void __launch_bounds__(kHeadThreads, 1) head_proj_kernel(const __grid
             const bool v_ok = v < P.v_end;
             const int n0 = tn * P.BN;
             const uint32_t taddr = tmem_base + (static_cast<uint32_t>(lane_base) << 16) + static_cast<uint32_t>(ab * P.BN);
-            for (int c = 0; c < P.BN; c += 16) {
-                uint32_t r[16];
-                tmem_ld_32x16(taddr + c, r);
-                tmem_ld_wait();
-                if (v_ok) {
+            if (P.pairs == 0) {
+                for (int c = 0; c < P.BN; c += 16) {
+                    uint32_t r[16];
+                    tmem_ld_32x16(taddr + c, r);
+                    tmem_ld_wait();
+                    if (v_ok) {
 #pragma unroll
-                    for (int j = 0; j < 16; ++j) {
-                        const int n = n0 + c + j;
-                        if (n < P.M) P.logits[static_cast<size_t>(n) * P.V + v] = __uint_as_float(r[j]);
+                        for (int j = 0; j < 16; ++j) {
+                            const int n = n0 + c + j;
+                            if (n < P.M) P.logits[static_cast<size_t>(n) * P.V + v] = __uint_as_float(r[j]);
+                        }
+                    }
+                }
+            } else {
+                const int half = P.BN / 2;  // a multiple of 16
+                const bool unit_T = P.temperature == 1.0f;
+                for (int c = 0; c < half; c += 16) {
+                    uint32_t rc[16], ru[16];
+                    tmem_ld_32x16(taddr + c, rc);
+                    tmem_ld_32x16(taddr + half + c, ru);
+                    tmem_ld_wait();
+                    if (v_ok) {
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) {
+                            const int pair = tn * half + c + j;
+                            const float lc = __uint_as_float(rc[j]), lu = __uint_as_float(ru[j]);
+                            float g = __fmaf_rn(P.cfg_scale, __fsub_rn(lc, lu), lu);
+                            if (!unit_T) g = __fdiv_rn(g, P.temperature);
+                            if (pair < P.pairs) P.logits[static_cast<size_t>(pair) * P.V + v] = g;
+                        }
                     }
                 }
             }
@@ -197,8 +234,11 @@ __global__ void __launch_bounds__(kHeadThreads, 1) head_proj_kernel(const __grid
 
 }  // namespace
 
-extern "C" hawk_status hawk_head_proj(const void *x, const void *w, float *logits, int M, int hidden, int V,
-                                      int v_begin, int v_end, int32_t *dev_status, hawk_stream_t stream)
+namespace {
+// pairs == 0: logits [M][V]; pairs > 0: M == 2 * pairs and `logits` receives guided rows [pairs][V].
+hawk_status head_proj_impl(const void *x, const void *w, float *logits, int M, int pairs, float cfg_scale,
+                           float temperature, int hidden, int V, int v_begin, int v_end, int32_t *dev_status,
+                           hawk_stream_t stream)
 {
     if (M < 0 || hidden < 0 || V < 0) return HAWK_ERR_SHAPE;
     if (v_begin < 0 || v_end > V || v_begin > v_end) return HAWK_ERR_SHAPE;
@@ -216,9 +256,21 @@ extern "C" hawk_status hawk_head_proj(const void *x, const void *w, float *logit
     P.V = V;
     P.v_begin = v_begin;
     P.v_end = v_end;
-    P.tiles_n = (M + 255) / 256;
-    const int per_tile = (M + P.tiles_n - 1) / P.tiles_n;
-    P.BN = (per_tile + 15) / 16 * 16;
+    P.pairs = pairs;
+    P.cfg_scale = cfg_scale;
+    P.temperature = temperature;
+    int x_box_rows;
+    if (pairs == 0) {
+        P.tiles_n = (M + 255) / 256;
+        const int per_tile = (M + P.tiles_n - 1) / P.tiles_n;
+        P.BN = (per_tile + 15) / 16 * 16;
+        x_box_rows = P.BN;
+    } else {  // half a tile of conditional rows, half of unconditional ones; each half a multiple of 16
+        P.tiles_n = (pairs + 127) / 128;
+        const int per_tile = (pairs + P.tiles_n - 1) / P.tiles_n;
+        x_box_rows = (per_tile + 15) / 16 * 16;
+        P.BN = 2 * x_box_rows;
+    }
     P.tiles_m = (v_end - v_begin + kBM - 1) / kBM;
     P.stage_bytes = kATileBytes + P.BN * kBK * 2;
     const int smem_budget = 200 * 1024;
@@ -232,7 +284,7 @@ extern "C" hawk_status hawk_head_proj(const void *x, const void *w, float *logit
     if (!hawk_host::encode_bf16_rows_sw128(&map_w, w, static_cast<uint64_t>(V), static_cast<uint64_t>(hidden), kBM,
                                            true) ||
         !hawk_host::encode_bf16_rows_sw128(&map_x, x, static_cast<uint64_t>(M), static_cast<uint64_t>(hidden),
-                                           static_cast<uint32_t>(P.BN), true))
+                                           static_cast<uint32_t>(x_box_rows), true))
         return HAWK_ERR_CUDA;
 
     // always ask for enough shared memory that a second block cannot share the SM: each block owns all of TMEM
@@ -250,4 +302,25 @@ extern "C" hawk_status hawk_head_proj(const void *x, const void *w, float *logit
     const cudaError_t err = hawk_host::launch_dependent(head_proj_kernel, dim3(grid), dim3(kHeadThreads), smem_req,
                                                         reinterpret_cast<cudaStream_t>(stream), map_w, map_x, P);
     return err == cudaSuccess ? HAWK_OK : HAWK_ERR_CUDA;
+}
+}  // namespace
+
+extern "C" hawk_status hawk_head_proj(const void *x, const void *w, float *logits, int M, int hidden, int V,
+                                      int v_begin, int v_end, int32_t *dev_status, hawk_stream_t stream)
+{
+    return head_proj_impl(x, w, logits, M, 0, 1.0f, 1.0f, hidden, V, v_begin, v_end, dev_status, stream);
+}
+
+extern "C" hawk_status hawk_head_proj_cfg(const void *x, const void *w, float *guided, int B, int rows, int hidden,
+                                          int V, int v_begin, int v_end, float cfg_scale, float temperature,
+                                          int32_t *dev_status, hawk_stream_t stream)
+{
+    if (B < 0 || rows < 0) return HAWK_ERR_SHAPE;
+    if (static_cast<long long>(B) * rows > (1 << 29)) return HAWK_ERR_UNSUPPORTED;
+    if (!(temperature == temperature) || !(cfg_scale == cfg_scale) || isinf(temperature) || isinf(cfg_scale) ||
+        !(temperature > 0.f))
+        return HAWK_ERR_PARAM;
+    const int pairs = B * rows;
+    return head_proj_impl(x, w, guided, 2 * pairs, pairs, cfg_scale, temperature, hidden, V, v_begin, v_end, dev_status,
+                          stream);
 }
