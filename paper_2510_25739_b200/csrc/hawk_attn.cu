@@ -74,6 +74,7 @@ struct AttnParams {
     int tiles_per_item;   // tiles of the longest admissible prefix: ceil((max_prefix_len + K) / kTileKeys)
     int workers;          // warps that own a share of the flat tile list
     long long total_tiles;  // items * tiles_per_item
+    int idx32;              // (total_tiles + 1) * workers fits 31 bits: the merge kernel may index in 32 bits
     float scale_log2;     // sm_scale * log2(e)
     int32_t *dev_status;
 };
@@ -510,52 +511,174 @@ __global__ void __launch_bounds__(kWarps * 32, 1) attn_kernel(const __grid_const
     if (flags && lane == 0 && P.dev_status) atomicOr(P.dev_status, flags);
 }
 
+// Division of a 31-bit unsigned number by a divisor fixed at launch: one multiply-high and a shift
+// (division by invariant integers, Granlund and Montgomery): mul = ceil(2^(31 + ceil(log2 d)) / d),
+// n / d = umulhi(n, mul) >> (ceil(log2 d) - 1) for 0 <= n < 2^31.  The host fills it in.
+struct FastDiv {
+    uint32_t d, mul, shr;
+    __host__ void set(uint32_t div)
+    {
+        d = div;
+        if (div <= 1) {
+            mul = 0;
+            shr = 0;
+            return;
+        }
+        uint32_t lg = 0;
+        while ((1u << lg) < div) ++lg;  // ceil(log2 div), 1..31
+        const unsigned long long pw = 1ull << (31 + lg);
+        mul = static_cast<uint32_t>((pw + div - 1) / div);
+        shr = lg - 1;
+    }
+    __device__ __forceinline__ uint32_t div(uint32_t n) const { return d <= 1 ? n : __umulhi(n, mul) >> shr; }
+    __device__ __forceinline__ uint32_t divmod(uint32_t n, uint32_t &rem) const
+    {
+        const uint32_t q = div(n);
+        rem = n - q * d;
+        return q;
+    }
+};
+
+// Divisors of the merge kernel's index arithmetic.
+struct MergeDivs {
+    FastDiv workers, total, tiles_per_item, chunks, h_kv, rows_per_item, k;
+};
+
+// Index arithmetic of the merge kernel: which item a unit stands for, the shares its tiles went to and
+// where their partial results are.  Two forms: 32-bit with launch-time divisors when every product of
+// a tile index and the worker count fits 31 bits (a dozen divisions by run-time values would otherwise
+// be most of the kernel's instructions), plain 64-bit otherwise.
+template <int AHEAD>
+struct MergeIndex {
+    bool cut;  // this unit stands for an item whose tiles were spread over several shares
+    int item, g_first, g_last, s, hk, chunk;
+    int seg_off[AHEAD];  // first tile, inside the item, of contribution t
+    int slot_id[AHEAD];  // its partial slot: share * 2 + (0 head of the share, 1 tail)
+};
+
+template <int AHEAD>
+__device__ __forceinline__ void merge_index32(const AttnParams &P, const MergeDivs &dv, int unit, int units,
+                                              int by_boundary, MergeIndex<AHEAD> &ix)
+{
+    const uint32_t T = static_cast<uint32_t>(P.total_tiles), W = static_cast<uint32_t>(P.workers);
+    const uint32_t tpi = static_cast<uint32_t>(P.tiles_per_item);
+    auto begin_of = [&](uint32_t g) { return dv.workers.div(g * T); };
+    auto owner_of = [&](uint32_t f) { return dv.total.div((f + 1) * W - 1); };
+    uint32_t item = static_cast<uint32_t>(unit);
+    bool first_inside = true;
+    if (by_boundary && unit < units) {
+        const uint32_t sb = begin_of(static_cast<uint32_t>(unit) + 1);
+        item = dv.tiles_per_item.div(sb);
+        const uint32_t ia = item * tpi;
+        first_inside = sb > ia && (unit == 0 || begin_of(static_cast<uint32_t>(unit)) <= ia);
+    }
+    ix.cut = unit < units && first_inside;
+    ix.item = static_cast<int>(item);
+    ix.g_first = ix.g_last = ix.s = ix.hk = ix.chunk = 0;
+    const uint32_t a = item * tpi, b = a + tpi;
+    if (ix.cut) {
+        ix.g_first = static_cast<int>(owner_of(a));
+        ix.g_last = static_cast<int>(owner_of(b - 1));
+        uint32_t chunk, hk;
+        const uint32_t it = dv.chunks.divmod(item, chunk);
+        ix.s = static_cast<int>(dv.h_kv.divmod(it, hk));
+        ix.hk = static_cast<int>(hk);
+        ix.chunk = static_cast<int>(chunk);
+        ix.cut = ix.g_first != ix.g_last;
+    }
+#pragma unroll
+    for (int t = 0; t < AHEAD; ++t) {
+        const int gg = min(ix.g_first + t, ix.g_last);
+        const uint32_t sb = begin_of(static_cast<uint32_t>(gg));
+        ix.seg_off[t] = static_cast<int>((sb > a ? sb : a) - a);
+        ix.slot_id[t] = gg * 2 + (a <= sb ? 0 : 1);
+    }
+}
+
+template <int AHEAD>
+__device__ __forceinline__ void merge_index64(const AttnParams &P, int unit, int units, int by_boundary,
+                                              MergeIndex<AHEAD> &ix)
+{
+    const long long T = P.total_tiles, tpi = P.tiles_per_item;
+    long long item = unit;
+    bool first_inside = true;
+    if (by_boundary && unit < units) {
+        const long long sb = share_begin(unit + 1, T, P.workers);
+        item = sb / tpi;
+        const long long ia = item * tpi;
+        first_inside = sb > ia && (unit == 0 || share_begin(unit, T, P.workers) <= ia);
+    }
+    ix.cut = unit < units && first_inside;
+    ix.item = static_cast<int>(item);
+    ix.g_first = ix.g_last = ix.s = ix.hk = ix.chunk = 0;
+    const long long a = item * tpi, b = a + tpi;
+    if (ix.cut) {
+        ix.g_first = owner(a, T, P.workers);
+        ix.g_last = owner(b - 1, T, P.workers);
+        int it = ix.item;
+        ix.chunk = it % P.chunks;
+        it /= P.chunks;
+        ix.hk = it % P.H_kv;
+        ix.s = it / P.H_kv;
+        ix.cut = ix.g_first != ix.g_last;
+    }
+#pragma unroll
+    for (int t = 0; t < AHEAD; ++t) {
+        const int gg = min(ix.g_first + t, ix.g_last);
+        const long long sb = share_begin(gg, T, P.workers);
+        ix.seg_off[t] = static_cast<int>((sb > a ? sb : a) - a);
+        ix.slot_id[t] = gg * 2 + (a <= sb ? 0 : 1);
+    }
+}
+
 // Merges the partial results of every item whose tiles were spread over several shares:
 // one warp per (item, query row of the item), lanes across the head dimension.  All index
-// arithmetic comes before the wait on the attention kernel; after it the loads of up to kAhead
-// contributions are issued together, so the kernel adds one memory round trip to the call.
-template <int D>
-__global__ void attn_combine_kernel(const AttnParams P, int items, int rows_per_item)
+// arithmetic and the loads of the call's inputs come before the wait on the attention kernel; after
+// it the loads of up to kAhead contributions are issued together, so the kernel adds one memory
+// round trip to the call.
+// The grid runs over `units`: the items themselves, or (by_boundary) the share boundaries 1 .. workers-1
+// when there are fewer of those than items; a boundary stands for the item it falls into, if it is the
+// first one strictly inside that item, so every cut item is merged exactly once and the grid stays
+// within one wave however many items the call has.
+// kAhead = 2 (an item never spans more than two shares: the common case when items are shorter than
+// shares) keeps the kernel within 32 registers, so that eight blocks fit an SM and the grid is one wave.
+template <int D, int kAhead>
+__global__ void __launch_bounds__(256, kAhead <= 2 ? 8 : 4)
+    attn_combine_kernel(const AttnParams P, const MergeDivs dv, int units, int by_boundary)
 {
     constexpr int TK = AttnCfg<D>::kTileKeys;
     constexpr int PER = D / 32;
-    constexpr int kAhead = 4;
     allow_dependent_launch();
     const int wid = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const int lane = threadIdx.x & 31;
-    const int item = wid / rows_per_item, r = wid - item * rows_per_item;
+    uint32_t r_u;
+    const int unit = static_cast<int>(dv.rows_per_item.divmod(static_cast<uint32_t>(wid), r_u));
+    const int r = static_cast<int>(r_u);
     const long long T = P.total_tiles;
-    const long long a = static_cast<long long>(item) * P.tiles_per_item, b = a + P.tiles_per_item;
-    bool active = item < items;
-    int g_first = 0, g_last = 0, s = 0, hk = 0, chunk = 0;
+    MergeIndex<kAhead> ix;
+    if (P.idx32)  // block-uniform
+        merge_index32<kAhead>(P, dv, unit, units, by_boundary, ix);
+    else
+        merge_index64<kAhead>(P, unit, units, by_boundary, ix);
+    const long long a = static_cast<long long>(ix.item) * P.tiles_per_item;
+    const int g_first = ix.g_first, g_last = ix.g_last, s = ix.s, hk = ix.hk, chunk = ix.chunk;
     const int group = P.H / P.H_kv;
-    if (active) {
-        g_first = owner(a, T, P.workers);
-        g_last = owner(b - 1, T, P.workers);
-        int it = item;
-        chunk = it % P.chunks;
-        it /= P.chunks;
-        hk = it % P.H_kv;
-        s = it / P.H_kv;
-        // one share held the whole item and wrote the result itself; rows past the item's last do not exist
-        active = g_first != g_last && r < min(P.rows_per_item, group * P.K - chunk * P.rows_per_item);
-    }
+    // one share held the whole item and wrote the result itself; rows past the item's last do not exist
+    const bool active = ix.cut && r < min(P.rows_per_item, group * P.K - chunk * P.rows_per_item);
     // tile offset inside the item at which each contribution starts, and where it is stored
     const float *slot[kAhead];
     int seg_off[kAhead];
 #pragma unroll
     for (int t = 0; t < kAhead; ++t) {
-        const int gg = min(g_first + t, g_last);
-        const long long sb = share_begin(gg, T, P.workers);
-        seg_off[t] = static_cast<int>((sb > a ? sb : a) - a);
-        slot[t] = P.part + (static_cast<size_t>(gg) * 2 + (a <= sb ? 0 : 1)) * P.rows_per_item * (D + 2);
+        seg_off[t] = ix.seg_off[t];
+        slot[t] = P.part + static_cast<size_t>(ix.slot_id[t]) * P.rows_per_item * (D + 2);
     }
+    const int pl_raw = active ? P.prefix_len[s] : 0;  // an input of the call: readable before the wait
     grid_dependency_wait();  // every thread waits, so this grid cannot retire before the attention kernel has
     if (!active) return;
 
     float2 ml[kAhead];
     float v[kAhead][PER];
-    const int pl_raw = P.prefix_len[s];
 #pragma unroll
     for (int t = 0; t < kAhead; ++t) {  // slots always exist; which of them were written is decided below
         ml[t] = *reinterpret_cast<const float2 *>(slot[t] + P.rows_per_item * D + 2 * r);
@@ -603,7 +726,8 @@ __global__ void attn_combine_kernel(const AttnParams P, int items, int rows_per_
     }
     const float inv = 1.f / ll;
     const int gr = chunk * P.rows_per_item + r;
-    const int h = hk * group + gr / P.K, i = gr % P.K;
+    uint32_t i_u;
+    const int h = hk * group + static_cast<int>(dv.k.divmod(static_cast<uint32_t>(gr), i_u)), i = static_cast<int>(i_u);
     __nv_bfloat16 *dst = P.out + ((static_cast<size_t>(s) * P.K + i) * P.H + h) * D + lane * PER;
 #pragma unroll
     for (int c = 0; c < PER; c += 2)
@@ -734,6 +858,7 @@ hawk_status verify_attn_impl(const void *q, const void *k_cache, const void *v_c
     P.tiles_per_item = pl.tiles_per_item;
     P.workers = pl.workers;
     P.total_tiles = pl.total_tiles;
+    P.idx32 = (pl.total_tiles + 1) * pl.workers < (1ll << 31) ? 1 : 0;
     P.scale_log2 = sm_scale * 1.4426950408889634f;
     P.dev_status = dev_status;
 
@@ -753,12 +878,24 @@ hawk_status verify_attn_impl(const void *q, const void *k_cache, const void *v_c
     if (err != cudaSuccess) return HAWK_ERR_CUDA;
     if (pl.any_cut) {
         const int threads = 256;
-        const long long warps = static_cast<long long>(pl.items) * pl.rows_per_item;
+        const int by_boundary = pl.items > pl.workers - 1 ? 1 : 0;
+        const int units = by_boundary ? pl.workers - 1 : pl.items;
+        const long long warps = static_cast<long long>(units) * pl.rows_per_item;
         const int blocks = static_cast<int>((warps * 32 + threads - 1) / threads);
-        err = D == 64 ? hawk_host::launch_dependent(attn_combine_kernel<64>, dim3(blocks), dim3(threads), 0, st, P,
-                                                    pl.items, pl.rows_per_item)
-                      : hawk_host::launch_dependent(attn_combine_kernel<128>, dim3(blocks), dim3(threads), 0, st, P,
-                                                    pl.items, pl.rows_per_item);
+        MergeDivs dv;
+        dv.workers.set(static_cast<uint32_t>(pl.workers));
+        dv.total.set(P.idx32 ? static_cast<uint32_t>(pl.total_tiles) : 1u);
+        dv.tiles_per_item.set(static_cast<uint32_t>(pl.tiles_per_item));
+        dv.chunks.set(static_cast<uint32_t>(pl.chunks));
+        dv.h_kv.set(static_cast<uint32_t>(P.H_kv));
+        dv.rows_per_item.set(static_cast<uint32_t>(pl.rows_per_item));
+        dv.k.set(static_cast<uint32_t>(P.K));
+        // shares hold floor(T / workers) tiles or one more: an item no longer than the shorter kind meets at
+        // most one share boundary
+        const bool two = pl.tiles_per_item <= pl.total_tiles / pl.workers;
+        auto kernel = D == 64 ? (two ? attn_combine_kernel<64, 2> : attn_combine_kernel<64, 4>)
+                              : (two ? attn_combine_kernel<128, 2> : attn_combine_kernel<128, 4>);
+        err = hawk_host::launch_dependent(kernel, dim3(blocks), dim3(threads), 0, st, P, dv, units, by_boundary);
         if (err != cudaSuccess) return HAWK_ERR_CUDA;
     }
     return HAWK_OK;
