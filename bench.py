@@ -45,8 +45,8 @@ L2_BYTES = 126 * 1024 * 1024
 # DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) of one hawk_verify_attn call, attention kernel
 # plus merge kernel, from the ncu capture summarised in profiles/; None where no capture of the
 # current kernels exists for that workload.
-ATTN_TRAFFIC_BYTES = {2: 94_461_000 + 3_286_000 + 2_044_000,   # attention read + write, merge kernel read
-                      5: 679_408_000 + 4_214_000}               # attention kernel alone (merge kernel not captured)
+ATTN_TRAFFIC_BYTES = {2: 94_459_000 + 3_156_000 + 2_048_000,     # attention read + write, merge kernel read
+                      5: 679_418_000 + 4_810_000 + 4_756_000}
 
 
 def measured_peaks():
