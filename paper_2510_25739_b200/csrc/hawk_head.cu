@@ -44,6 +44,49 @@ struct HeadParams {
     int32_t *dev_status;
 };
 
+// Epilogue of one tile for one thread: the thread owns token id v (its tensor-memory lane) and walks
+// the tile's token columns 16 at a time; lanes of a warp hold consecutive ids, so every store
+// instruction writes 128 contiguous bytes of one logits row.
+// Warps that share a lane quarter split the 16-column chunks among themselves (chunk0, chunk_step).
+__device__ __forceinline__ void epilogue_store(const HeadParams &P, uint32_t taddr, int tn, int v, bool v_ok,
+                                               int chunk0 = 0, int chunk_step = 1)
+{
+    if (P.pairs == 0) {
+        const int n0 = tn * P.BN;
+        for (int c = 16 * chunk0; c < P.BN; c += 16 * chunk_step) {
+            uint32_t r[16];
+            tmem_ld_32x16(taddr + c, r);
+            tmem_ld_wait();
+            if (v_ok) {
+#pragma unroll
+                for (int j = 0; j < 16; ++j) {
+                    const int n = n0 + c + j;
+                    if (n < P.M) P.logits[static_cast<size_t>(n) * P.V + v] = __uint_as_float(r[j]);
+                }
+            }
+        }
+    } else {
+        const int half = P.BN / 2;  // a multiple of 16
+        const bool unit_T = P.temperature == 1.0f;
+        for (int c = 16 * chunk0; c < half; c += 16 * chunk_step) {
+            uint32_t rc[16], ru[16];
+            tmem_ld_32x16(taddr + c, rc);
+            tmem_ld_32x16(taddr + half + c, ru);
+            tmem_ld_wait();
+            if (v_ok) {
+#pragma unroll
+                for (int j = 0; j < 16; ++j) {
+                    const int pair = tn * half + c + j;
+                    const float lc = __uint_as_float(rc[j]), lu = __uint_as_float(ru[j]);
+                    float g = __fmaf_rn(P.cfg_scale, __fsub_rn(lc, lu), lu);
+                    if (!unit_T) g = __fdiv_rn(g, P.temperature);
+                    if (pair < P.pairs) P.logits[static_cast<size_t>(pair) * P.V + v] = g;
+                }
+            }
+        }
+    }
+}
+
 __global__ void __launch_bounds__(kHeadThreads, 1) head_proj_kernel(const __grid_constant__ CUtensorMap map_w,
                                                                     const __grid_constant__ CUtensorMap map_x,
                                                                     const HeadParams P)
@@ -179,41 +222,8 @@ __global__ void __launch_bounds__(kHeadThreads, 1) head_proj_kernel(const __grid
             tcgen05_fence_after();
             const int v = P.v_begin + tm * kBM + lane_base + lane;  // this thread's token id
             const bool v_ok = v < P.v_end;
-            const int n0 = tn * P.BN;
             const uint32_t taddr = tmem_base + (static_cast<uint32_t>(lane_base) << 16) + static_cast<uint32_t>(ab * P.BN);
-            if (P.pairs == 0) {
-                for (int c = 0; c < P.BN; c += 16) {
-                    uint32_t r[16];
-                    tmem_ld_32x16(taddr + c, r);
-                    tmem_ld_wait();
-                    if (v_ok) {
-#pragma unroll
-                        for (int j = 0; j < 16; ++j) {
-                            const int n = n0 + c + j;
-                            if (n < P.M) P.logits[static_cast<size_t>(n) * P.V + v] = __uint_as_float(r[j]);
-                        }
-                    }
-                }
-            } else {
-                const int half = P.BN / 2;  // a multiple of 16
-                const bool unit_T = P.temperature == 1.0f;
-                for (int c = 0; c < half; c += 16) {
-                    uint32_t rc[16], ru[16];
-                    tmem_ld_32x16(taddr + c, rc);
-                    tmem_ld_32x16(taddr + half + c, ru);
-                    tmem_ld_wait();
-                    if (v_ok) {
-#pragma unroll
-                        for (int j = 0; j < 16; ++j) {
-                            const int pair = tn * half + c + j;
-                            const float lc = __uint_as_float(rc[j]), lu = __uint_as_float(ru[j]);
-                            float g = __fmaf_rn(P.cfg_scale, __fsub_rn(lc, lu), lu);
-                            if (!unit_T) g = __fdiv_rn(g, P.temperature);
-                            if (pair < P.pairs) P.logits[static_cast<size_t>(pair) * P.V + v] = g;
-                        }
-                    }
-                }
-            }
+            epilogue_store(P, taddr, tn, v, v_ok);
             tcgen05_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(&acc_empty[ab]);
@@ -229,6 +239,181 @@ __global__ void __launch_bounds__(kHeadThreads, 1) head_proj_kernel(const __grid
     if (warp == 1) {
         tcgen05_fence_after();
         tmem_dealloc(tmem_base, kTmemCols);
+    }
+}
+
+
+// ------------------------------------------------------------------------------------------------
+// The same projection by pairs of CTAs (clusters of two) that drive one MMA of 256 token ids x BN
+// token rows together (tcgen05 cta_group::2).  Each CTA of a pair loads its own 128 weight rows and
+// only HALF of the tile's token rows; the tensor cores of both SMs read both halves.  Per flop a CTA
+// moves two thirds of the shared-memory bytes of the single-CTA kernel (fills and operand reads), which
+// is what bounds that kernel once there are enough token rows to be tensor-bound.
+//   warp 0      TMA producer (own weight rows, own half of the token rows), in both CTAs
+//   warp 1      rank 0: issues the pair MMAs and commits to the barriers of both CTAs
+//               (both CTAs' loads count on rank 0's stage barrier)
+//   warps 2..9  epilogue of the CTA's own 128 accumulator rows, in both CTAs: two warps per lane
+//               quarter, taking alternate 16-column chunks
+// Tensor memory is allocated and freed by warp 1 of each CTA of the pair.
+#ifndef HAWK_PAIR_TMEM_COLS
+#define HAWK_PAIR_TMEM_COLS 512
+#endif
+constexpr uint32_t kPairTmemCols = HAWK_PAIR_TMEM_COLS;
+
+constexpr int kPairThreads = 320;  // producer, MMA, and two epilogue warps per tensor-memory lane quarter
+
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kPairThreads, 1)
+    head_proj_pair_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_x,
+                          const HeadParams P)
+{
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    uint64_t *full_bar = reinterpret_cast<uint64_t *>(smem + static_cast<size_t>(P.stages) * P.stage_bytes);
+    uint64_t *empty_bar = full_bar + kMaxStages;
+    uint64_t *acc_full = empty_bar + kMaxStages;   // [2]
+    uint64_t *acc_empty = acc_full + 2;            // [2], used in rank 0: 4 epilogue warps of each CTA
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(acc_empty + 2);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const uint32_t rank = cluster_cta_rank();
+    const int pair = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
+    hawk::allow_dependent_launch();
+    const int kblocks = P.hidden / kBK;
+    const int total_tiles = P.tiles_m * P.tiles_n;
+    const int half_n = P.BN / 2;
+
+    if (tid == 0) {
+        for (int i = 0; i < P.stages; ++i) {
+            mbar_init(&full_bar[i], 1);
+            mbar_init(&empty_bar[i], 1);
+        }
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(&acc_full[i], 1);
+            mbar_init(&acc_empty[i], 16);  // 8 epilogue warps in each CTA
+        }
+        *abort_flag = 0;
+        fence_mbar_init();
+    }
+    if (warp == 1) {
+        tmem_alloc_pair(tmem_slot, kPairTmemCols);
+        tmem_relinquish_pair();
+    }
+    tcgen05_fence_before();
+    __syncthreads();
+    cluster_sync_all();  // the other CTA's barriers exist before anything is signalled across
+    tcgen05_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+    grid_dependency_wait();
+
+    if (warp == 0) {
+        // =========================== TMA producer (both CTAs)
+        if (lane == 0) {
+            prefetch_tensormap(&map_w);
+            prefetch_tensormap(&map_x);
+            const uint32_t tx_bytes = static_cast<uint32_t>(P.stage_bytes);
+            int st = 0;
+            uint32_t ph = 0;
+            bool ok = true;
+            for (int tile = pair; tile < total_tiles && ok; tile += n_pairs) {
+                const int tn = tile % P.tiles_n, tm = tile / P.tiles_n;
+                const int row_w = P.v_begin + tm * (2 * kBM) + static_cast<int>(rank) * kBM;
+                const int row_x = P.pairs == 0 ? tn * P.BN + static_cast<int>(rank) * half_n
+                                               : (rank == 0 ? tn * half_n : P.pairs + tn * half_n);
+                for (int kb = 0; kb < kblocks; ++kb) {
+                    ok = mbar_wait_cluster(&empty_bar[st], ph ^ 1u, abort_flag);
+                    if (!ok) break;
+                    uint8_t *a = smem + static_cast<size_t>(st) * P.stage_bytes;
+                    if (rank == 0) mbar_arrive_expect_tx(&full_bar[st], 2 * tx_bytes);  // both CTAs' halves
+                    const uint32_t bar0 = map_shared_to_cta(&full_bar[st], 0);
+                    tma_load_2d_pair(a, &map_w, kb * kBK, row_w, bar0);
+                    tma_load_2d_pair(a + kATileBytes, &map_x, kb * kBK, row_x, bar0);
+                    if (++st == P.stages) {
+                        st = 0;
+                        ph ^= 1u;
+                    }
+                }
+            }
+            if (!ok) {
+                *abort_flag = 1;
+                if (P.dev_status) atomicOr(P.dev_status, HAWK_DEV_TIMEOUT);
+            }
+        }
+    } else if (warp == 1 && rank != 0) {
+        // rank 1's warp 1 only allocates and frees tensor memory
+    } else if (warp == 1) {
+        // =========================== rank 0: MMA issuer for the pair
+        if (lane == 0) {
+            const uint32_t idesc = umma_idesc_bf16_f32(2 * kBM, P.BN);
+            int st = 0;
+            uint32_t ph = 0;
+            bool ok = true;
+            int it = 0;
+            for (int tile = pair; tile < total_tiles && ok; tile += n_pairs, ++it) {
+                const int ab = it & 1;
+                const uint32_t acc_ph = (it >> 1) & 1;
+                ok = mbar_wait_cluster(&acc_empty[ab], acc_ph ^ 1u, abort_flag);  // both epilogues drained it
+                if (!ok) break;
+                tcgen05_fence_after();
+                const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(ab * P.BN);
+                for (int kb = 0; kb < kblocks; ++kb) {
+                    ok = mbar_wait_cluster(&full_bar[st], ph, abort_flag);  // both CTAs' halves have landed
+                    if (!ok) break;
+                    tcgen05_fence_after();
+                    const uint32_t a_addr = smem_u32(smem + static_cast<size_t>(st) * P.stage_bytes);
+                    const uint64_t da = umma_desc_k_major_sw128(a_addr);
+                    const uint64_t db = umma_desc_k_major_sw128(a_addr + kATileBytes);
+#pragma unroll
+                    for (int k = 0; k < kBK / 16; ++k)
+                        umma_bf16_pair(d_tmem, da + static_cast<uint64_t>(2 * k), db + static_cast<uint64_t>(2 * k), idesc,
+                                       (kb | k) != 0 ? 1u : 0u);
+                    umma_commit_pair(&empty_bar[st], 3);  // the stage is reusable in both CTAs
+                    if (++st == P.stages) {
+                        st = 0;
+                        ph ^= 1u;
+                    }
+                }
+                if (!ok) break;
+                umma_commit_pair(&acc_full[ab], 3);  // accumulator complete, in both CTAs
+            }
+            if (!ok) {
+                *abort_flag = 1;
+                if (P.dev_status) atomicOr(P.dev_status, HAWK_DEV_TIMEOUT);
+            }
+        }
+    } else {
+        // =========================== epilogue warps (both CTAs): own TMEM lanes 32*(warp%4) .. +31
+        const int lane_base = (warp & 3) * 32;
+        const uint32_t acc_empty_rank0[2] = {map_shared_to_cta(&acc_empty[0], 0), map_shared_to_cta(&acc_empty[1], 0)};
+        bool ok = true;
+        int it = 0;
+        for (int tile = pair; tile < total_tiles && ok; tile += n_pairs, ++it) {
+            const int tn = tile % P.tiles_n, tm = tile / P.tiles_n;
+            const int ab = it & 1;
+            const uint32_t acc_ph = (it >> 1) & 1;
+            ok = mbar_wait_cluster(&acc_full[ab], acc_ph, abort_flag);
+            if (!ok) break;
+            tcgen05_fence_after();
+            const int v = P.v_begin + tm * (2 * kBM) + static_cast<int>(rank) * kBM + lane_base + lane;
+            const bool v_ok = v < P.v_end;
+            const uint32_t taddr = tmem_base + (static_cast<uint32_t>(lane_base) << 16) + static_cast<uint32_t>(ab * P.BN);
+            epilogue_store(P, taddr, tn, v, v_ok, (warp - 2) >> 2, 2);
+            tcgen05_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive_cluster(acc_empty_rank0[ab]);
+        }
+        if (!ok && lane == 0) {
+            *abort_flag = 1;
+            if (P.dev_status) atomicOr(P.dev_status, HAWK_DEV_TIMEOUT);
+        }
+    }
+
+    tcgen05_fence_before();
+    __syncthreads();
+    cluster_sync_all();  // neither CTA frees tensor memory or exits while the other may still use or signal it
+    if (warp == 1) {
+        tcgen05_fence_after();
+        tmem_dealloc_pair(tmem_base, kPairTmemCols);
     }
 }
 
@@ -259,20 +444,30 @@ hawk_status head_proj_impl(const void *x, const void *w, float *logits, int M, i
     P.pairs = pairs;
     P.cfg_scale = cfg_scale;
     P.temperature = temperature;
+    // From HAWK_HEAD_PAIR_MIN_ROWS token rows on, pairs of CTAs share a tile (cta_group::2).  Measured: with
+    // 1024 rows the pair kernel takes 42 us where the single-CTA kernel takes 45; with 384 rows they tie; below
+    // that the call is bound by the weight stream and the single-CTA kernel, with twice as many tiles, is ahead.
+#ifndef HAWK_HEAD_PAIR_MIN_ROWS
+#define HAWK_HEAD_PAIR_MIN_ROWS 512
+#endif
+    const bool use_pair = M >= HAWK_HEAD_PAIR_MIN_ROWS && sm_count >= 2;
+    const int max_bn = use_pair ? static_cast<int>(kPairTmemCols) / 2 : 256;  // two accumulators in tensor memory
+    const int bn_step = use_pair ? 32 : 16;  // a pair's tile splits into two halves of a multiple of 16 rows
     int x_box_rows;
     if (pairs == 0) {
-        P.tiles_n = (M + 255) / 256;
+        P.tiles_n = (M + max_bn - 1) / max_bn;
         const int per_tile = (M + P.tiles_n - 1) / P.tiles_n;
-        P.BN = (per_tile + 15) / 16 * 16;
-        x_box_rows = P.BN;
+        P.BN = (per_tile + bn_step - 1) / bn_step * bn_step;
+        x_box_rows = use_pair ? P.BN / 2 : P.BN;
     } else {  // half a tile of conditional rows, half of unconditional ones; each half a multiple of 16
-        P.tiles_n = (pairs + 127) / 128;
+        P.tiles_n = (pairs + max_bn / 2 - 1) / (max_bn / 2);
         const int per_tile = (pairs + P.tiles_n - 1) / P.tiles_n;
         x_box_rows = (per_tile + 15) / 16 * 16;
         P.BN = 2 * x_box_rows;
     }
-    P.tiles_m = (v_end - v_begin + kBM - 1) / kBM;
-    P.stage_bytes = kATileBytes + P.BN * kBK * 2;
+    const int tile_rows = use_pair ? 2 * kBM : kBM;  // token ids per tile
+    P.tiles_m = (v_end - v_begin + tile_rows - 1) / tile_rows;
+    P.stage_bytes = kATileBytes + x_box_rows * kBK * 2 * (pairs != 0 && !use_pair ? 2 : 1);
     const int smem_budget = 200 * 1024;
     int stages = smem_budget / P.stage_bytes;
     if (stages > kMaxStages) stages = kMaxStages;
@@ -288,19 +483,46 @@ hawk_status head_proj_impl(const void *x, const void *w, float *logits, int M, i
         return HAWK_ERR_CUDA;
 
     // always ask for enough shared memory that a second block cannot share the SM: each block owns all of TMEM
-    const size_t smem_bytes = 1024 + static_cast<size_t>(stages) * P.stage_bytes + (2 * kMaxStages + 4) * 8 + 64;
+    const size_t smem_bytes = 1024 + static_cast<size_t>(stages) * P.stage_bytes + (3 * kMaxStages + 4) * 8 + 64;
     const size_t smem_req = smem_bytes < 120 * 1024 ? 120 * 1024 : smem_bytes;
-    static bool attr_done = false;
-    if (!attr_done) {
+    int device = 0;
+    if (cudaGetDevice(&device) != cudaSuccess || device < 0 || device >= 64) return HAWK_ERR_CUDA;
+    static unsigned long long attr_done = 0;  // per device: the dynamic shared memory limit is a per-device attribute
+    if (!((attr_done >> device) & 1ull)) {
         if (cudaFuncSetAttribute(head_proj_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) !=
-            cudaSuccess)
+                cudaSuccess ||
+            cudaFuncSetAttribute(head_proj_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) !=
+                cudaSuccess)
             return HAWK_ERR_CUDA;
-        attr_done = true;
+        attr_done |= 1ull << device;
     }
     const int total_tiles = P.tiles_m * P.tiles_n;
-    const int grid = total_tiles < sm_count ? total_tiles : sm_count;
-    const cudaError_t err = hawk_host::launch_dependent(head_proj_kernel, dim3(grid), dim3(kHeadThreads), smem_req,
-                                                        reinterpret_cast<cudaStream_t>(stream), map_w, map_x, P);
+    cudaError_t err;
+    if (use_pair) {
+        // pairs that can be resident at once (an SM without a free neighbour in its group takes none): a
+        // persistent grid larger than that would run its last pairs after all the others have finished
+        static int max_pairs_of[64];
+        if (max_pairs_of[device] == 0) {
+            cudaLaunchConfig_t occ = {};
+            occ.gridDim = dim3(sm_count / 2 * 2);
+            occ.blockDim = dim3(kPairThreads);
+            occ.dynamicSmemBytes = 227 * 1024 - 1024;
+            int n = 0;
+            if (cudaOccupancyMaxActiveClusters(&n, head_proj_pair_kernel, &occ) != cudaSuccess || n < 1) {
+                (void)cudaGetLastError();
+                n = sm_count / 4;  // conservative: half of the SMs
+            }
+            max_pairs_of[device] = n < sm_count / 2 ? n : sm_count / 2;
+        }
+        const int max_pairs = max_pairs_of[device];
+        const int n_pairs = total_tiles < max_pairs ? total_tiles : max_pairs;
+        err = hawk_host::launch_dependent(head_proj_pair_kernel, dim3(2 * n_pairs), dim3(kPairThreads), smem_req,
+                                          reinterpret_cast<cudaStream_t>(stream), map_w, map_x, P);
+    } else {
+        const int grid = total_tiles < sm_count ? total_tiles : sm_count;
+        err = hawk_host::launch_dependent(head_proj_kernel, dim3(grid), dim3(kHeadThreads), smem_req,
+                                          reinterpret_cast<cudaStream_t>(stream), map_w, map_x, P);
+    }
     return err == cudaSuccess ? HAWK_OK : HAWK_ERR_CUDA;
 }
 }  // namespace

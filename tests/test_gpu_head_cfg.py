@@ -42,6 +42,8 @@ CASES = [
     (13, 10, 192, 384, 0, 384, 0.0, 2.0),        # 130 pairs: two token tiles, the second nearly empty
     (30, 10, 320, 700, 1, 699, 3.0, 1.0),        # 300 pairs: three token tiles
     (3, 22, 1024, 2048, 0, 2048, 3.0, 1.0),      # tree-shaped rows, more k-blocks than stages
+    (32, 8, 256, 1024, 0, 1024, 3.0, 1.0),       # 256 pairs = 512 rows: the CTA-pair kernel, two tiles of 128 pairs
+    (40, 9, 128, 700, 5, 690, 7.5, 0.9),         # 360 pairs: CTA pairs, three ragged tiles
 ]
 
 
