@@ -597,19 +597,26 @@ def bench_tree(cfg, stream, torch, hawk, peaks, seed, branching=(3, 2, 2)):
         for t in sets:
             lens.append(run(t))
         stream.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=stream):
+            for t in sets:
+                run(t)
+        for _ in range(3):
+            g.replay()
+        stream.synchronize()
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        n = 60
+        n = 20
         e0.record(stream)
-        for i in range(n):
-            run(sets[i % n_rep])
+        for _ in range(n):
+            g.replay()
         e1.record(stream)
         stream.synchronize()
-    us = e0.elapsed_time(e1) * 1e3 / n
+    us = e0.elapsed_time(e1) * 1e3 / (n * n_rep)
     nbytes = 2 * B * N * row_bytes
     return {"us": us, "tree": f"branching {branching}, {N} nodes, {NQ} draft rows per sequence", "rows": B * N,
             "logit_bytes": nbytes, "GB/s": nbytes / us / 1e3, "frac_hbm": nbytes / us / 1e3 / peaks["hbm_gbs"],
             "mean_accept_len": float(torch.stack(lens).float().mean().item()),
-            "timing": "eager launches back to back (includes launch overhead), replicas rotating"}
+            "timing": "graph of back-to-back calls, replicas rotating"}
 
 
 def bench_pool(cfg, stream, torch, hawk, peaks, seed, IW=32, VSD=2, K=3, branching=(3, 2, 2)):
