@@ -71,6 +71,20 @@ def test_small_cases(V, vb, ve, top_k, K, B, bonus):
     assert res["exempt_accept"] + res["exempt_resample"] <= B
 
 
+@pytest.mark.parametrize("V,vb,ve,top_k,K,B,bonus", [
+    (1000, 4, 996, 50, 5, 40, False),      # 200 rows of 992 ids
+    (4096, 0, 4096, 300, 4, 50, True),     # 250 rows (bonus row included), a full 256-thread block per row
+    (8192, 8, 8000, 0, 3, 60, False),      # 180 rows, no top-k, 512-thread blocks
+    (16384, 0, 16384, 2000, 2, 160, False),  # 320 rows on 148 SMs: three waves
+    (1001, 0, 1001, 50, 5, 40, False),     # rows that are not 16-byte aligned
+])
+def test_more_rows_than_sms(V, vb, ve, top_k, K, B, bonus):
+    """Calls with more rows than SMs: several waves of one-row blocks."""
+    cfg = wl.config(2, B=B, K=K, V=V, v_begin=vb, v_end=ve, top_k=top_k, cfg_scale=3.0, H=4, H_kv=4)
+    res, _ = _run_case(cfg, 91 + V + K, has_bonus=bonus)
+    assert res["exempt_accept"] + res["exempt_resample"] <= max(2, B // 4)
+
+
 @pytest.mark.parametrize("config_id", [1, 2, 3, 4, 5])
 def test_configs_full_size(config_id):
     cfg = wl.config(config_id)
