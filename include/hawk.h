@@ -165,6 +165,10 @@ hawk_status hawk_head_proj(const void *x, const void *w, float *logits, int M, i
  *               normal use (p never leaves the chip)
  *   workspace   at least hawk_cfg_accept_workspace_bytes(...) bytes, 16-byte aligned; needs no
  *               initialisation
+ * Every row is judged by a thread block of its own.  A call with more rows than the GPU runs at once
+ * lets the blocks of later positions look at the verdicts their sequence already has, and a row
+ * behind a rejection (step 5 never reads it) does no work; the results do not depend on it, and with
+ * p_debug every row is computed.
  * Supported: 1 <= K <= 16; 1 <= v_end - v_begin <= 32768 (one row is held in one
  * thread block's registers); temperature > 0.
  * Errors: NULL, SHAPE, ALIGN, UNSUPPORTED, WORKSPACE, PARAM (cfg_scale or temperature not finite,

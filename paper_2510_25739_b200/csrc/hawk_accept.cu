@@ -19,6 +19,8 @@
 
 #include <mutex>
 
+#include <climits>
+
 #include "hawk_common.cuh"
 
 namespace {
@@ -29,6 +31,7 @@ constexpr int kMaxRounds = 48;  // each narrowing round shrinks the value range 
 
 constexpr int ROW_ACCEPTED = -1;
 constexpr int ROW_REJECTED_NO_TOKEN = -2;  // rejected and nothing has positive mass
+constexpr int ROW_UNKNOWN = INT_MIN;       // no verdict yet (calls with more rows than SMs clear row_out to this)
 
 struct AcceptParams {
     const float *logits;
@@ -41,6 +44,7 @@ struct AcceptParams {
     int top_k;
     int vec_ok;
     int guided_in;     // logits is [B][rows][V] of guided logits instead of [2B][rows][V]
+    int skip_mode;     // row_out was cleared: a row whose sequence is known to be rejected earlier does nothing
     int32_t *row_out;  // [B][rows]
     float *p_debug;
     int32_t *dev_status;
@@ -498,6 +502,18 @@ __global__ void __launch_bounds__(NT) accept_rows_kernel(const AcceptParams P)
 
     const int row = blockIdx.x;  // position-major: all rows of position 0 first
     const int i = row / P.B, b = row - i * P.B;
+    // A chain ends at its first rejection, so the rows behind it are never looked at.  With more rows than SMs
+    // the blocks of the later positions start after those of the earlier ones have finished: such a block looks
+    // at the verdicts its sequence already has and, if one of them is a rejection, has nothing to do.  A verdict
+    // that is not visible yet only costs the skipped work; the result does not depend on what is seen here.
+    if (P.skip_mode && i > 0) {
+        int rejected = 0;
+        if (tid < i) {
+            const int c = *reinterpret_cast<const volatile int32_t *>(&P.row_out[b * P.rows + tid]);
+            rejected = (c != ROW_UNKNOWN && c != ROW_ACCEPTED) ? 1 : 0;
+        }
+        if (__syncthreads_or(rejected)) return;
+    }
     const bool bonus = (i == P.K);
     const int n = P.n;
     const bool vec_ok = P.vec_ok != 0;
@@ -837,6 +853,16 @@ __global__ void tree_walk_kernel(const int32_t *verdict, int B, int N, int max_d
 }
 
 // One thread per sequence: the first rejected row decides accept_len and the correction token.
+// Marks every row "no verdict yet".  Reads nothing that an earlier kernel writes, so the marking runs before
+// the dependency wait (alongside the tail of the preceding kernel); the wait keeps the stream's order.
+__global__ void accept_clear_kernel(int32_t *row_out, int n)
+{
+    hawk::allow_dependent_launch();
+    const int idx = blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx < n) row_out[idx] = ROW_UNKNOWN;
+    hawk::grid_dependency_wait();
+}
+
 __global__ void accept_finalize_kernel(const int32_t *row_out, int B, int K, int rows, int32_t *accept_len,
                                        int32_t *out_token)
 {
@@ -934,7 +960,16 @@ hawk_status cfg_accept_impl(const float *logits, int guided_in, const float *q_p
 
     cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
     const int grid = B * P.rows;
-    cudaError_t err;  // 16 ids per thread; the block as wide as the row needs
+    cudaError_t err;
+    // more rows than SMs: the later rows can see the verdicts of the earlier ones (see accept_rows_kernel)
+    int sm_count = 0;
+    (void)hawk_host::is_sm100(&sm_count);
+    P.skip_mode = (grid > sm_count + sm_count / 2 && !p_debug) ? 1 : 0;  // below 1.5 waves the marking costs more than it saves
+    if (P.skip_mode) {
+        err = hawk_host::launch_dependent(accept_clear_kernel, dim3((grid + 255) / 256), dim3(256), 0, st, P.row_out, grid);
+        if (err != cudaSuccess) return HAWK_ERR_CUDA;
+    }
+    // 16 ids per thread; the block as wide as the row needs
     if (n <= 4096) err = launch_rows<256, 4>(P, grid, st);
     else if (n <= 8192) err = launch_rows<512, 4>(P, grid, st);
     else if (n <= 16384) err = launch_rows<1024, 4>(P, grid, st);
