@@ -509,7 +509,7 @@ def main():
                  "frac_tensor": head_flops(cfg) / kernels["head"] / 1e6 / peaks["bf16_tflops"]},
         "accept": {"us": kernels["accept"], "GB/s": accept_bytes(cfg, cfg.B * cfg.K) / kernels["accept"] / 1e3,
                    "frac_hbm": accept_bytes(cfg, cfg.B * cfg.K) / kernels["accept"] / 1e3 / peaks["hbm_gbs"],
-                   "bytes_counted": "both logit rows of every position + one q row per position"},
+                   "bytes_counted": "both logit rows of every position + one q row per position (the definition's rows; in calls of more than 1.5 waves rows behind a known rejection are not read, so fewer bytes move)"},
         "mean_accept_len": mean_len, "sequences_with_rejection": rej, "q_rows_on_chain": q_rows,
         "two_call_form": {
             "what": "hawk_head_proj_cfg + hawk_cfg_accept_guided: one guided logits row per position crosses HBM",
