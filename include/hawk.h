@@ -212,8 +212,9 @@ hawk_status hawk_cfg_accept(const float *logits, const float *q_probs, const int
  *   out_token   int32 [B] (out)  correction token; -1 if the refined target has no mass at all
  *   path        optional int32 [B][max_depth] (out): accepted nodes in order, -1 beyond accept_len
  *   workspace   at least hawk_tree_accept_workspace_bytes(B, N) bytes, 16-byte aligned, no initialisation
- * Every node is judged by its own thread block whether or not the walk reaches it, so the cost is
- * B*N rows.  Supported: 1 <= N <= 65536; at most 16 children per node; valid ids as hawk_cfg_accept.
+ * Every node is judged by its own thread block, so the cost is at most B*N rows; in a call with more
+ * rows than the GPU runs at once, a node whose parent is already known not to have picked it does no
+ * work (the walk cannot reach it; the results do not depend on this).  Supported: 1 <= N <= 65536; at most 16 children per node; valid ids as hawk_cfg_accept.
  * A child range that breaks these rules is clamped and flagged HAWK_DEV_BAD_TREE; the walk always ends.
  * Errors: NULL, SHAPE, ALIGN, UNSUPPORTED, WORKSPACE, PARAM, CUDA.  B == 0 returns HAWK_OK.
  * ---------------------------------------------------------------------------------------------- */

@@ -641,6 +641,8 @@ struct TreeParams {
     int top_k;
     int vec_ok;
     int guided_in;     // logits is [B][N][V] of guided logits instead of [2B][N][V]
+    int skip_mode;     // verdicts were cleared and `parent` filled in: a node its parent did not pick does nothing
+    const int32_t *parent;  // [N], written by tree_prepare_kernel
     int32_t *verdict;  // [B][N]: >= 0 the child that passed; -1 stop without a token; <= -2 stop, token = -v - 2
     int32_t *dev_status;
 };
@@ -656,6 +658,23 @@ __global__ void __launch_bounds__(NT) tree_rows_kernel(const TreeParams P)
 
     const int row = blockIdx.x;  // node-major
     const int node = row / P.B, b = row - node * P.B;
+    // The walk reaches a node only as the child its parent picked.  With more rows than SMs the blocks of the
+    // deeper nodes start after their parents have finished: a node whose parent is known to have picked
+    // another child, to have stopped, or to be unreachable itself, is marked unreachable and does nothing.
+    if (P.skip_mode && node > 0) {
+        int dead = 0;
+        if (tid == 0) {
+            const int par = P.parent[node];
+            if (par >= 0 && par < node) {
+                const int v = *reinterpret_cast<const volatile int32_t *>(&P.verdict[b * P.N + par]);
+                dead = (v != ROW_UNKNOWN && v != node) ? 1 : 0;
+            }
+        }
+        if (__syncthreads_or(dead)) {
+            if (tid == 0) P.verdict[b * P.N + node] = -1;
+            return;
+        }
+    }
     const int n = P.n;
     const bool vec_ok = P.vec_ok != 0;
     const float *lc = P.logits + (static_cast<size_t>(b) * P.N + node) * P.V + P.v_begin;
@@ -821,6 +840,25 @@ __global__ void pool_scatter_kernel(const int32_t *row_token, const int32_t *nod
         tok = row_token[b * NQ + r];
     }
     node_token[idx] = tok;
+}
+
+// For calls with more rows than SMs: marks every verdict "unknown" and writes each node's parent (the
+// child ranges clamped exactly as tree_rows_kernel clamps them).
+__global__ void tree_prepare_kernel(int32_t *verdict, int32_t *parent, const int32_t *child_begin, int B, int N)
+{
+    hawk::allow_dependent_launch();
+    hawk::grid_dependency_wait();
+    const int idx = blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx < B * N) verdict[idx] = ROW_UNKNOWN;
+    if (idx == 0) parent[0] = -1;
+    if (idx < N) {
+        int cb = child_begin[idx], ce = child_begin[idx + 1];
+        if (cb < ce) {
+            cb = max(idx + 1, min(cb, N));
+            ce = max(cb, min(ce, min(N, cb + kMaxChildren)));
+            for (int c = cb; c < ce; ++c) parent[c] = idx;
+        }
+    }
 }
 
 // One thread per sequence: follows the verdicts from the root.
@@ -1009,7 +1047,7 @@ extern "C" hawk_status hawk_cfg_accept_guided(const float *guided, const float *
 extern "C" size_t hawk_tree_accept_workspace_bytes(int B, int N)
 {
     if (B <= 0 || N <= 0) return 0;
-    return static_cast<size_t>(B) * static_cast<size_t>(N) * sizeof(int32_t);
+    return (static_cast<size_t>(B) + 1) * static_cast<size_t>(N) * sizeof(int32_t);  // verdicts, then a parent per node
 }
 
 namespace {
@@ -1059,11 +1097,21 @@ hawk_status tree_accept_impl(const float *logits, int guided_in, const float *q_
     P.vec_ok = (V % 4 == 0 && v_begin % 4 == 0) ? 1 : 0;
     P.guided_in = guided_in;
     P.verdict = static_cast<int32_t *>(workspace);
+    int32_t *parent = P.verdict + static_cast<size_t>(B) * N;
+    P.parent = parent;
     P.dev_status = dev_status;
 
     cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
     const int grid = B * N;
     cudaError_t err;
+    int sm_count = 0;
+    (void)hawk_host::is_sm100(&sm_count);
+    P.skip_mode = grid > sm_count + sm_count / 2 ? 1 : 0;  // as in the chain: worth it from 1.5 waves on
+    if (P.skip_mode) {
+        err = hawk_host::launch_dependent(tree_prepare_kernel, dim3((grid + 255) / 256), dim3(256), 0, st, P.verdict, parent,
+                                          child_begin, B, N);
+        if (err != cudaSuccess) return HAWK_ERR_CUDA;
+    }
     if (n <= 4096) err = launch_tree_rows<256, 4>(P, grid, st);
     else if (n <= 8192) err = launch_tree_rows<512, 4>(P, grid, st);
     else if (n <= 16384) err = launch_tree_rows<1024, 4>(P, grid, st);

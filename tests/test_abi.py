@@ -140,7 +140,7 @@ def test_tree_accept_argument_checks(lib):
              depth=2, al=p, out=p, path=p, ws=p, wsb=1 << 20):
         return f(lg, q, tok, nq, cb, ua, ur, B, N, NQ, V, vb, ve, s, T, k, depth, al, out, path, ws, wsb, None, None)
 
-    assert lib.hawk_tree_accept_workspace_bytes(4, 22) == 4 * 22 * 4
+    assert lib.hawk_tree_accept_workspace_bytes(4, 22) == (4 + 1) * 22 * 4   # verdicts and one parent per node
     assert lib.hawk_tree_accept_workspace_bytes(0, 22) == 0
     assert call(B=0) == OK
     assert call(B=-1) == E_SHAPE and call(depth=-1) == E_SHAPE

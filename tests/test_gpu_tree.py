@@ -72,6 +72,8 @@ def _case(B, V, vb, ve, top_k, branching, seed, alpha=0.7, cfg_scale=3.0, expect
     (3, 65536, 4, 8196, 2000, (4, 1, 3)),
     (6, 20000, 0, 20000, 0, (2, 2)),
     (16, 16384, 0, 16384, 2000, (1, 1, 1, 1, 1)),       # a chain
+    (24, 4096, 0, 4096, 300, (3, 2, 2)),                # 528 rows: more than 1.5 waves, unreachable nodes do no work
+    (40, 1000, 4, 996, 50, (2, 2, 2)),                  # 600 narrow rows
 ])
 def test_matches_oracle(B, V, vb, ve, top_k, branching):
     res, ora = _case(B, V, vb, ve, top_k, branching, seed=300 + V + len(branching))
