@@ -892,9 +892,14 @@ hawk_status verify_attn_impl(const void *q, const void *k_cache, const void *v_c
         dv.k.set(static_cast<uint32_t>(P.K));
         // shares hold floor(T / workers) tiles or one more: an item no longer than the shorter kind meets at
         // most one share boundary
-        const bool two = pl.tiles_per_item <= pl.total_tiles / pl.workers;
-        auto kernel = D == 64 ? (two ? attn_combine_kernel<64, 2> : attn_combine_kernel<64, 4>)
-                              : (two ? attn_combine_kernel<128, 2> : attn_combine_kernel<128, 4>);
+        // shares hold floor(T / workers) tiles or one more: an item of t tiles meets at most ceil(t / floor) share
+        // boundaries, i.e. has at most that many contributions plus one; all of them are loaded at once
+        const long long min_share = pl.total_tiles / pl.workers;
+        const long long contrib = min_share > 0 ? (pl.tiles_per_item + min_share - 1) / min_share + 1 : 9;
+        auto kernel = D == 64 ? (contrib <= 2 ? attn_combine_kernel<64, 2>
+                                 : contrib <= 4 ? attn_combine_kernel<64, 4> : attn_combine_kernel<64, 8>)
+                              : (contrib <= 2 ? attn_combine_kernel<128, 2>
+                                 : contrib <= 4 ? attn_combine_kernel<128, 4> : attn_combine_kernel<128, 8>);
         err = hawk_host::launch_dependent(kernel, dim3(blocks), dim3(threads), 0, st, P, dv, units, by_boundary);
         if (err != cudaSuccess) return HAWK_ERR_CUDA;
     }
