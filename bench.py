@@ -45,6 +45,8 @@ L2_BYTES = 126 * 1024 * 1024
 # DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) of one hawk_verify_attn call, attention kernel
 # plus merge kernel, from the ncu capture summarised in profiles/; None where no capture of the
 # current kernels exists for that workload.
+NOMINAL_HBM_GBS = 7700.0       # HBM3e figure of the HGX B200 data sheet
+NOMINAL_BF16_TFLOPS = 2250.0   # dense bf16
 ATTN_TRAFFIC_BYTES = {2: 94_459_000 + 3_156_000 + 2_048_000,     # attention read + write, merge kernel read
                       5: 679_418_000 + 4_810_000 + 4_756_000}
 
@@ -452,6 +454,40 @@ def main():
             a1.record(stream)
             stream.synchronize()
             kernels[name] = a0.elapsed_time(a1) * 1e3 / (n * n_rep)   # us per launch
+        # the same three with ONE replica repeated: inputs L2-warm where they fit (labelled as such)
+        for name, fn in (("attn", run_attn), ("head", run_head), ("accept", run_accept)):
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=stream):
+                for _ in range(4):
+                    fn(cfg, first, hawk)
+            for _ in range(3):
+                g.replay()
+            stream.synchronize()
+            a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a0.record(stream)
+            for _ in range(20):
+                g.replay()
+            a1.record(stream)
+            stream.synchronize()
+            kernels[name + "_l2_warm"] = a0.elapsed_time(a1) * 1e3 / 80
+        # the head over ALL columns where only part of the vocabulary is valid (the 65536-entry vocabulary)
+        if cfg.V_valid < cfg.V:
+            full_logits = torch.zeros((cfg.M, cfg.V), dtype=torch.float32, device="cuda")
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=stream):
+                for r in reps:
+                    hawk.head_proj(r.x, r.w, 0, cfg.V, logits=full_logits, dev_status=r.status)
+            for _ in range(3):
+                g.replay()
+            stream.synchronize()
+            a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a0.record(stream)
+            for _ in range(10):
+                g.replay()
+            a1.record(stream)
+            stream.synchronize()
+            kernels["head_full_vocab"] = a0.elapsed_time(a1) * 1e3 / (10 * n_rep)
+            del full_logits
     # ---- the two-call form: guidance combined in the head's epilogue, accept reads one guided row per position
     for r in reps:
         r.guided = torch.zeros((cfg.B, cfg.K, cfg.V), dtype=torch.float32, device="cuda")
@@ -502,15 +538,28 @@ def main():
     q_rows = sum(int(r.accept_len.clamp(max=cfg.K - 1).add(1).sum().item()) for r in reps) / n_rep
     stage = {
         "attn": {"us": kernels["attn"], "GB/s": attn_bytes(cfg) / kernels["attn"] / 1e3,
-                 "frac_hbm": attn_bytes(cfg) / kernels["attn"] / 1e3 / peaks["hbm_gbs"]},
+                 "frac_hbm": attn_bytes(cfg) / kernels["attn"] / 1e3 / peaks["hbm_gbs"],
+                 "frac_hbm_nominal": attn_bytes(cfg) / kernels["attn"] / 1e3 / NOMINAL_HBM_GBS,
+                 "us_one_replica_l2_warm": kernels["attn_l2_warm"]},
         "head": {"us": kernels["head"], "GB/s": head_bytes(cfg) / kernels["head"] / 1e3,
                  "frac_hbm": head_bytes(cfg) / kernels["head"] / 1e3 / peaks["hbm_gbs"],
                  "TFLOP/s": head_flops(cfg) / kernels["head"] / 1e6,
-                 "frac_tensor": head_flops(cfg) / kernels["head"] / 1e6 / peaks["bf16_tflops"]},
+                 "frac_tensor": head_flops(cfg) / kernels["head"] / 1e6 / peaks["bf16_tflops"],
+                 "frac_hbm_nominal": head_bytes(cfg) / kernels["head"] / 1e3 / NOMINAL_HBM_GBS,
+                 "frac_tensor_nominal": head_flops(cfg) / kernels["head"] / 1e6 / NOMINAL_BF16_TFLOPS,
+                 "us_one_replica_l2_warm": kernels["head_l2_warm"]},
         "accept": {"us": kernels["accept"], "GB/s": accept_bytes(cfg, cfg.B * cfg.K) / kernels["accept"] / 1e3,
                    "frac_hbm": accept_bytes(cfg, cfg.B * cfg.K) / kernels["accept"] / 1e3 / peaks["hbm_gbs"],
+                   "frac_hbm_nominal": accept_bytes(cfg, cfg.B * cfg.K) / kernels["accept"] / 1e3 / NOMINAL_HBM_GBS,
+                   "us_one_replica_l2_warm": kernels["accept_l2_warm"],
                    "bytes_counted": "both logit rows of every position + one q row per position (the definition's rows; in calls of more than 1.5 waves rows behind a known rejection are not read, so fewer bytes move)"},
         "mean_accept_len": mean_len, "sequences_with_rejection": rej, "q_rows_on_chain": q_rows,
+        **({"head_full_vocab": {
+            "us": kernels["head_full_vocab"], "columns": cfg.V,
+            "TFLOP/s": 2.0 * cfg.M * cfg.hidden * cfg.V / kernels["head_full_vocab"] / 1e6,
+            "GB/s": (cfg.V * cfg.hidden * 2 + cfg.M * cfg.hidden * 2 + cfg.M * cfg.V * 4) / kernels["head_full_vocab"] / 1e3,
+            "frac_hbm": (cfg.V * cfg.hidden * 2 + cfg.M * cfg.hidden * 2 + cfg.M * cfg.V * 4)
+                        / kernels["head_full_vocab"] / 1e3 / peaks["hbm_gbs"]}} if "head_full_vocab" in kernels else {}),
         "two_call_form": {
             "what": "hawk_head_proj_cfg + hawk_cfg_accept_guided: one guided logits row per position crosses HBM",
             "head_cfg_us": kernels["head_cfg"], "accept_guided_us": kernels["accept_guided"],
