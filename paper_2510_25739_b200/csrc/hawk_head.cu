@@ -39,6 +39,7 @@ struct HeadParams {
     int tiles_n;   // token tiles
     int stages;
     int stage_bytes;
+    int ksplit;    // 1, or 2: two work units per tile, each over half of the hidden dimension (output zeroed first)
     int pairs;     // 0: plain logits; > 0: guided logits of this many (sequence, position) pairs
     float cfg_scale, temperature;
     int32_t *dev_status;
@@ -61,7 +62,11 @@ __device__ __forceinline__ void epilogue_store(const HeadParams &P, uint32_t tad
 #pragma unroll
                 for (int j = 0; j < 16; ++j) {
                     const int n = n0 + c + j;
-                    if (n < P.M) P.logits[static_cast<size_t>(n) * P.V + v] = __uint_as_float(r[j]);
+                    if (n < P.M) {
+                        float *dst = &P.logits[static_cast<size_t>(n) * P.V + v];
+                        if (P.ksplit == 1) *dst = __uint_as_float(r[j]);
+                        else atomicAdd(dst, __uint_as_float(r[j]));  // two addends onto zero: the order cannot matter
+                    }
                 }
             }
         }
@@ -103,7 +108,9 @@ __global__ void __launch_bounds__(kHeadThreads, 1) head_proj_kernel(const __grid
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     hawk::allow_dependent_launch();
     const int kblocks = P.hidden / kBK;
-    const int total_tiles = P.tiles_m * P.tiles_n;
+    // a unit of work is a tile, or (ksplit == 2) one half of a tile's k-blocks; the halves add their results
+    const int total_tiles = P.tiles_m * P.tiles_n * P.ksplit;
+    const int kb_half = (kblocks + P.ksplit - 1) / P.ksplit;
 
     if (tid == 0) {
         for (int i = 0; i < P.stages; ++i) {
@@ -138,9 +145,11 @@ __global__ void __launch_bounds__(kHeadThreads, 1) head_proj_kernel(const __grid
             bool ok = true;
             long long issued = 0;
             for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
-                const int tn = tile % P.tiles_n, tm = tile / P.tiles_n;
+                const int part = tile % P.ksplit, t2 = tile / P.ksplit;
+                const int tn = t2 % P.tiles_n, tm = t2 / P.tiles_n;
                 const int row_w = P.v_begin + tm * kBM, row_x = tn * P.BN;
-                for (int kb = 0; kb < kblocks; ++kb) {
+                const int kb0 = part * kb_half, kb1 = min(kblocks, kb0 + kb_half);
+                for (int kb = kb0; kb < kb1; ++kb) {
                     ok = mbar_wait(&empty_bar[st], ph ^ 1u, abort_flag);
                     if (!ok) break;
                     uint8_t *a = smem + static_cast<size_t>(st) * P.stage_bytes;
@@ -181,7 +190,9 @@ __global__ void __launch_bounds__(kHeadThreads, 1) head_proj_kernel(const __grid
                 if (!ok) break;
                 tcgen05_fence_after();
                 const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(ab * P.BN);
-                for (int kb = 0; kb < kblocks; ++kb) {
+                const int part = tile % P.ksplit;
+                const int kb0 = part * kb_half, kb1 = min(kblocks, kb0 + kb_half);
+                for (int kb = kb0; kb < kb1; ++kb) {
                     ok = mbar_wait(&full_bar[st], ph, abort_flag);
                     if (!ok) break;
                     tcgen05_fence_after();
@@ -192,7 +203,7 @@ __global__ void __launch_bounds__(kHeadThreads, 1) head_proj_kernel(const __grid
                     for (int k = 0; k < kBK / 16; ++k) {
                         // 16 bf16 along K = 32 bytes = 2 units of the descriptor's 16-byte address field
                         umma_bf16(d_tmem, da + static_cast<uint64_t>(2 * k), db + static_cast<uint64_t>(2 * k), idesc,
-                                  (kb | k) != 0 ? 1u : 0u);
+                                  ((kb - kb0) | k) != 0 ? 1u : 0u);
                     }
                     umma_commit(&empty_bar[st]);  // stage reusable once these MMAs have read it
                     if (++st == P.stages) {
@@ -214,7 +225,8 @@ __global__ void __launch_bounds__(kHeadThreads, 1) head_proj_kernel(const __grid
         bool ok = true;
         int it = 0;
         for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++it) {
-            const int tn = tile % P.tiles_n, tm = tile / P.tiles_n;
+            const int t2 = tile / P.ksplit;
+            const int tn = t2 % P.tiles_n, tm = t2 / P.tiles_n;
             const int ab = it & 1;
             const uint32_t acc_ph = (it >> 1) & 1;
             ok = mbar_wait(&acc_full[ab], acc_ph, abort_flag);
@@ -417,6 +429,18 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kPairThreads, 1)
     }
 }
 
+
+// Zeroes logits[M][v_begin, v_end) ahead of a call whose tiles are split along the hidden dimension.
+__global__ void head_zero_kernel(float *logits, int M, int V, int v_begin, int n)
+{
+    hawk::allow_dependent_launch();
+    hawk::grid_dependency_wait();
+    const long long idx = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x;
+    if (idx >= static_cast<long long>(M) * n) return;
+    const int m = static_cast<int>(idx / n), c = static_cast<int>(idx - static_cast<long long>(m) * n);
+    logits[static_cast<size_t>(m) * V + v_begin + c] = 0.f;
+}
+
 }  // namespace
 
 namespace {
@@ -496,8 +520,19 @@ hawk_status head_proj_impl(const void *x, const void *w, float *logits, int M, i
             return HAWK_ERR_CUDA;
         attr_done |= 1ull << device;
     }
-    const int total_tiles = P.tiles_m * P.tiles_n;
+    // few tiles and a long hidden dimension (a narrow valid range of a wide model): split every tile's k-blocks
+    // over two blocks so that twice as many SMs stream the weights; plain logits only (the guidance combine
+    // of the other form is applied to complete sums)
+    P.ksplit = (!use_pair && pairs == 0 && 2 * P.tiles_m * P.tiles_n <= sm_count && hidden / kBK >= 16) ? 2 : 1;
+    const int total_tiles = P.tiles_m * P.tiles_n * P.ksplit;
     cudaError_t err;
+    if (P.ksplit > 1) {
+        const int n = v_end - v_begin;
+        const long long cells = static_cast<long long>(M) * n;
+        err = hawk_host::launch_dependent(head_zero_kernel, dim3(static_cast<unsigned>((cells + 255) / 256)), dim3(256), 0,
+                                          reinterpret_cast<cudaStream_t>(stream), logits, M, V, v_begin, n);
+        if (err != cudaSuccess) return HAWK_ERR_CUDA;
+    }
     if (use_pair) {
         // pairs that can be resident at once (an SM without a free neighbour in its group takes none): a
         // persistent grid larger than that would run its last pairs after all the others have finished

@@ -43,7 +43,8 @@ SMALL = [
     (40, 256, 1000, 4, 996),       # range not aligned to the tile
     (100, 512, 520, 130, 400),
     (300, 256, 384, 0, 384),       # two token tiles
-    (17, 1024, 2048, 0, 2048),     # more k-blocks than pipeline stages
+    (17, 1024, 2048, 0, 2048),     # more k-blocks than pipeline stages; few tiles: each split over two blocks along hidden
+    (48, 1088, 1000, 4, 996),      # split along hidden with an odd number of k-blocks (17), ragged range
     (600, 320, 700, 1, 699),       # three token tiles, ragged both ways (from 512 rows on: the CTA-pair kernel)
     (512, 128, 256, 0, 256),       # CTA pairs: one tile of 256 ids x 256 rows per pair, two token tiles
     (1000, 192, 900, 3, 897),      # CTA pairs: ragged 256-id tiles, four token tiles of 256 rows (the last ragged)
