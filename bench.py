@@ -47,8 +47,8 @@ L2_BYTES = 126 * 1024 * 1024
 # current kernels exists for that workload.
 NOMINAL_HBM_GBS = 7700.0       # HBM3e figure of the HGX B200 data sheet
 NOMINAL_BF16_TFLOPS = 2250.0   # dense bf16
-ATTN_TRAFFIC_BYTES = {2: 94_459_000 + 3_156_000 + 2_048_000,     # attention read + write, merge kernel read
-                      5: 679_418_000 + 4_810_000 + 4_756_000}
+ATTN_TRAFFIC_BYTES = {2: 94_462_000 + 3_671_000 + 2_053_000,     # attention read + write, merge kernel read
+                      5: 679_406_000 + 5_353_000 + 4_757_000}
 
 
 def measured_peaks():
@@ -340,7 +340,13 @@ def main():
     n_rep = min(n_rep, 64)
     reps = [first] + [Replica(cfg, 1000 * cid + 17 * rank + 101 * i, torch, hawk) for i in range(1, n_rep)]
     stream = torch.cuda.Stream()
-    launches_per_step = (2 if first.attn_split else 1) + 1 + 2
+    # kernels per step: attention (+ its merge kernel when items are cut), head (+ a zeroing kernel when its tiles
+    # are split along the hidden dimension), accept rows + finalize (+ a marking kernel from 1.5 waves of rows on)
+    sms = torch.cuda.get_device_properties(local_rank).multi_processor_count
+    head_tiles = -(-cfg.V_valid // 128) * -(-cfg.M // 256)
+    head_split = cfg.M < 512 and 2 * head_tiles <= sms and cfg.hidden // 64 >= 16
+    accept_marks = cfg.B * cfg.K > sms + sms // 2
+    launches_per_step = (2 if first.attn_split else 1) + (2 if head_split else 1) + (3 if accept_marks else 2)
 
     # ---- one CUDA graph per replica: [ev0] attn [ev1] head accept
     graphs, evs = [], []
