@@ -891,14 +891,14 @@ __global__ void tree_walk_kernel(const int32_t *verdict, int B, int N, int max_d
 }
 
 // One thread per sequence: the first rejected row decides accept_len and the correction token.
-// Marks every row "no verdict yet".  Reads nothing that an earlier kernel writes, so the marking runs before
-// the dependency wait (alongside the tail of the preceding kernel); the wait keeps the stream's order.
+// Marks every row "no verdict yet" (after the dependency wait: the workspace may be memory that the preceding
+// kernel in the stream still uses).
 __global__ void accept_clear_kernel(int32_t *row_out, int n)
 {
     hawk::allow_dependent_launch();
+    hawk::grid_dependency_wait();
     const int idx = blockIdx.x * blockDim.x + threadIdx.x;
     if (idx < n) row_out[idx] = ROW_UNKNOWN;
-    hawk::grid_dependency_wait();
 }
 
 __global__ void accept_finalize_kernel(const int32_t *row_out, int B, int K, int rows, int32_t *accept_len,
