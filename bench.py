@@ -602,7 +602,7 @@ def main():
     }
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         _, t1, _ = oracle_sample(cfg, wl.seed_for(cid), 1)
-        reps_cpu = max(1, min(2000, int(15.0 / max(t1, 1e-3))))    # about 15 s of CPU work
+        reps_cpu = max(1, min(2000, int(22.0 / max(t1, 1e-3))))    # 10 to 30 s of CPU work (the first, cold step is the slowest)
         v, dt, cores = oracle_sample(cfg, wl.seed_for(cid), reps_cpu)
         line["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle",
                                 "sample": f"{reps_cpu} full steps of the workload ({dt:.1f} s)"}
