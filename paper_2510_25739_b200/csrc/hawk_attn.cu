@@ -42,6 +42,7 @@ using namespace hawk;
 //           Taken when the items fit (at most 3 per SM) and an item is short enough for one warp.
 constexpr int kWarpsShares = HAWK_ATTN_WARPS, kStagesShares = 3;
 constexpr int kWarpsWhole = 3, kStagesWhole = 8;
+constexpr int kWarpsGroup = 4, kStagesGroup = 2;  // blocks of 4 warps, three per SM: an item's 4 warps merge in shared memory
 constexpr int kWholeMaxTiles = 12;       // longest item (in tiles) that one warp takes alone: a lone warp needs
                                          // 0.75 us per tile, so beyond this the shares (and their merge) win
 constexpr int kStageBytes = HAWK_ATTN_STAGE_KB * 1024;  // K and V tile of one stage
@@ -56,7 +57,8 @@ struct AttnCfg {
     static_assert(2 * kHalves * kSubTileBytes == kStageBytes, "stage = K tile + V tile");
     static constexpr size_t smem_bytes(int warps, int stages)
     {
-        return 1024 /*align slack*/ + static_cast<size_t>(warps) * stages * kStageBytes + warps * stages * sizeof(uint64_t);
+        return 1024 /*align slack*/ + static_cast<size_t>(warps) * stages * kStageBytes + warps * stages * sizeof(uint64_t) +
+               64 /*one flag per warp: the warp left a partial result in its ring (group mode)*/;
     }
 };
 
@@ -74,6 +76,8 @@ struct AttnParams {
     int tiles_per_item;   // tiles of the longest admissible prefix: ceil((max_prefix_len + K) / kTileKeys)
     int workers;          // warps that own a share of the flat tile list
     long long total_tiles;  // items * tiles_per_item
+    int group_g;            // > 0: every item is split evenly over this many warps of one block, merged in shared memory
+    int items;              // items in the call
     int idx32;              // (total_tiles + 1) * workers fits 31 bits: the merge kernel may index in 32 bits
     float scale_log2;     // sm_scale * log2(e)
     int32_t *dev_status;
@@ -154,7 +158,7 @@ __device__ __forceinline__ uint32_t movmatrix_trans(uint32_t x)
 
 // NQT = number of 8-query column tiles of an item: rows_per_item / 8 (1..4 at D = 64, 1..3 at D = 128).
 template <int D, int NQT, int kWarps, int kStages>
-__global__ void __launch_bounds__(kWarps * 32, 1) attn_kernel(const __grid_constant__ CUtensorMap map_k,
+__global__ void __launch_bounds__(kWarps * 32, kWarps == kWarpsGroup ? 3 : 1) attn_kernel(const __grid_constant__ CUtensorMap map_k,
                                                            const __grid_constant__ CUtensorMap map_v,
                                                            const AttnParams P)
 {
@@ -165,12 +169,14 @@ __global__ void __launch_bounds__(kWarps * 32, 1) attn_kernel(const __grid_const
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     uint64_t *bars = reinterpret_cast<uint64_t *>(smem + kWarps * kStages * kStageBytes);
+    volatile int *has_part = reinterpret_cast<volatile int *>(bars + kWarps * kStages);  // [kWarps], group mode
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     // No allow_dependent_launch() here: with the merge kernel's blocks resident and waiting from the
     // start, this kernel measured 10 % slower; the merge kernel is released when the blocks exit.
     if (tid == 0) {
         for (int i = 0; i < kWarps * kStages; ++i) mbar_init(&bars[i], 1);
+        for (int i = 0; i < kWarps; ++i) has_part[i] = 0;
         fence_mbar_init();
         fence_proxy_async();
     }
@@ -180,13 +186,15 @@ __global__ void __launch_bounds__(kWarps * 32, 1) attn_kernel(const __grid_const
     // shares: the warps of a block take neighbouring shares; whole: items are dealt out to the blocks in turn
     const int w = kWarps == kWarpsWhole ? warp * static_cast<int>(gridDim.x) + static_cast<int>(blockIdx.x)
                                         : static_cast<int>(blockIdx.x) * kWarps + warp;
-    if (w >= P.workers) return;
+    const bool grouped = kWarps == kWarpsGroup && P.group_g > 0;
+    const bool idle = w >= P.workers;
+    if (idle && !grouped) return;  // (a grouped block meets again at the end: its idle warps walk an empty share)
     uint8_t *ring = smem + warp * kStages * kStageBytes;
     uint64_t *full_bar = bars + warp * kStages;
     const uint32_t ring_u32 = smem_u32(ring);
 
     const long long T = P.total_tiles;
-    const long long f_begin = share_begin(w, T, P.workers), f_end = share_begin(w + 1, T, P.workers);
+    const long long f_begin = idle ? 0 : share_begin(w, T, P.workers), f_end = idle ? 0 : share_begin(w + 1, T, P.workers);
     int flags = 0;
 
     uint64_t policy = 0;
@@ -285,7 +293,10 @@ __global__ void __launch_bounds__(kWarps * 32, 1) attn_kernel(const __grid_const
             }
         } else {
             const int slot = seg_start == f_begin ? 0 : 1;
-            float *ps = P.part + (static_cast<size_t>(w) * 2 + slot) * P.rows_per_item * (D + 2);
+            // grouped: the warp's ring is free by now (every copy issued has been consumed) and takes the partial
+            float *ps = grouped ? reinterpret_cast<float *>(ring)
+                                : P.part + (static_cast<size_t>(w) * 2 + slot) * P.rows_per_item * (D + 2);
+            if (grouped && lane == 0) has_part[warp] = 1;
 #pragma unroll
             for (int nq = 0; nq < NQT; ++nq)
 #pragma unroll
@@ -509,6 +520,49 @@ __global__ void __launch_bounds__(kWarps * 32, 1) attn_kernel(const __grid_const
         }
     }
     if (flags && lane == 0 && P.dev_status) atomicOr(P.dev_status, flags);
+
+    if (grouped) {
+        // ---- the G warps of an item sit side by side in this block: fold their partial results, in share
+        // order, straight from shared memory (no workspace, no merge kernel)
+        __syncthreads();
+        constexpr int PER = D / 32;
+        const int G = P.group_g, ipb = kWarps / G;
+        const int total = ipb * P.rows_per_item;
+        for (int idx = warp; idx < total; idx += kWarps) {
+            const int il = idx / P.rows_per_item, r = idx - il * P.rows_per_item;
+            const int item = static_cast<int>(blockIdx.x) * ipb + il;
+            if (item >= P.items) break;
+            int it = item;
+            const int chunk = it % P.chunks;
+            it /= P.chunks;
+            const int hk = it % P.H_kv, s = it / P.H_kv;
+            if (r >= min(P.rows_per_item, group * P.K - chunk * P.rows_per_item)) continue;
+            float acc[PER];
+#pragma unroll
+            for (int c = 0; c < PER; ++c) acc[c] = 0.f;
+            float mm = -CUDART_INF_F, ll = 0.f;
+            for (int gg = 0; gg < G; ++gg) {
+                const int wg = il * G + gg;
+                if (!has_part[wg]) continue;  // that share lay past the stream's last visible key
+                const float *ps = reinterpret_cast<const float *>(smem + wg * kStages * kStageBytes);
+                const float2 m_l = *reinterpret_cast<const float2 *>(ps + P.rows_per_item * D + 2 * r);
+                const float mn = fmaxf(mm, m_l.x);
+                const float mu = mn == -CUDART_INF_F ? 0.f : mn;
+                const float f_old = fast_exp2(mm - mu), f_new = fast_exp2(m_l.x - mu);
+                mm = mn;
+                ll = ll * f_old + m_l.y * f_new;
+#pragma unroll
+                for (int c = 0; c < PER; ++c) acc[c] = acc[c] * f_old + ps[r * D + lane * PER + c] * f_new;
+            }
+            const float inv = 1.f / ll;
+            const int gr = chunk * P.rows_per_item + r;
+            const int h = hk * group + gr / P.K, i = gr % P.K;
+            __nv_bfloat16 *dst = P.out + ((static_cast<size_t>(s) * P.K + i) * P.H + h) * D + lane * PER;
+#pragma unroll
+            for (int c = 0; c < PER; c += 2)
+                *reinterpret_cast<__nv_bfloat162 *>(dst + c) = __floats2bfloat162_rn(acc[c] * inv, acc[c + 1] * inv);
+        }
+    }
 }
 
 // Division of a 31-bit unsigned number by a divisor fixed at launch: one multiply-high and a shift
@@ -737,6 +791,7 @@ __global__ void __launch_bounds__(256, kAhead <= 2 ? 8 : 4)
 struct AttnPlan {
     int chunks, items, rows_per_item, tiles_per_item, workers, grid;
     bool whole;  // one warp per item (3 warps x 8 stages per block) instead of equal shares (8 x 3)
+    int group_g;  // > 0: every item split evenly over this many warps of a 4-warp block and merged there
     long long total_tiles;
     bool any_cut;  // some item's tiles are spread over more than one share: partials + merge kernel needed
 };
@@ -755,16 +810,27 @@ AttnPlan make_plan(int S, int K, int H, int H_kv, int D, int max_prefix_len)
     pl.tiles_per_item = (max_prefix_len + K + tk - 1) / tk;
     pl.total_tiles = static_cast<long long>(pl.items) * pl.tiles_per_item;
     pl.whole = pl.items <= kPlanSms * kWarpsWhole && pl.tiles_per_item <= kWholeMaxTiles;
+    // few long items of one 8-row column tile (a kernel of under 170 registers, three 4-warp blocks per SM): split
+    // each evenly over the 4 warps of a block if all blocks are resident at once; the warps fold their partial
+    // results in shared memory and nothing is left for a merge kernel
+    pl.group_g = 0;
+    if (pl.rows_per_item == 8 && pl.items <= 3 * kPlanSms && pl.tiles_per_item >= 2 * kWarpsGroup) {
+        pl.group_g = kWarpsGroup;
+        pl.whole = false;  // (from 8 tiles on, four warps with a merge in shared memory beat one warp alone)
+    }
     if (pl.whole) {
         pl.workers = pl.items;  // share g = item g
         pl.grid = pl.items < kPlanSms ? pl.items : kPlanSms;
+    } else if (pl.group_g > 0) {
+        pl.workers = pl.items * pl.group_g;  // share w = part (w % G) of item (w / G)
+        pl.grid = (pl.workers + kWarpsGroup - 1) / kWarpsGroup;
     } else {
         const long long cap = static_cast<long long>(kPlanSms) * kWarpsShares;
         pl.workers = static_cast<int>(pl.total_tiles < cap ? pl.total_tiles : cap);
         pl.grid = (pl.workers + kWarpsShares - 1) / kWarpsShares;
     }
     pl.any_cut = false;
-    for (int it = 0; it < pl.items && !pl.any_cut; ++it) {
+    for (int it = 0; it < pl.items && !pl.any_cut && pl.group_g == 0; ++it) {
         const long long a = static_cast<long long>(it) * pl.tiles_per_item, b = a + pl.tiles_per_item;
         pl.any_cut = owner(a, pl.total_tiles, pl.workers) != owner(b - 1, pl.total_tiles, pl.workers);
     }
@@ -791,6 +857,7 @@ template <int D, int NQT>
 cudaError_t launch_attn(const CUtensorMap &map_k, const CUtensorMap &map_v, const AttnParams &P, int grid, bool whole,
                         cudaStream_t st)
 {
+    if (P.group_g > 0) return launch_attn_shape<D, NQT, kWarpsGroup, kStagesGroup>(map_k, map_v, P, grid, st);
     return whole ? launch_attn_shape<D, NQT, kWarpsWhole, kStagesWhole>(map_k, map_v, P, grid, st)
                  : launch_attn_shape<D, NQT, kWarpsShares, kStagesShares>(map_k, map_v, P, grid, st);
 }
@@ -858,6 +925,8 @@ hawk_status verify_attn_impl(const void *q, const void *k_cache, const void *v_c
     P.tiles_per_item = pl.tiles_per_item;
     P.workers = pl.workers;
     P.total_tiles = pl.total_tiles;
+    P.group_g = pl.group_g;
+    P.items = pl.items;
     P.idx32 = (pl.total_tiles + 1) * pl.workers < (1ll << 31) ? 1 : 0;
     P.scale_log2 = sm_scale * 1.4426950408889634f;
     P.dev_status = dev_status;
