@@ -814,7 +814,10 @@ AttnPlan make_plan(int S, int K, int H, int H_kv, int D, int max_prefix_len)
     // each evenly over the 4 warps of a block if all blocks are resident at once; the warps fold their partial
     // results in shared memory and nothing is left for a merge kernel
     pl.group_g = 0;
-    if (pl.rows_per_item == 8 && pl.items <= 3 * kPlanSms && pl.tiles_per_item >= 2 * kWarpsGroup) {
+    // (with fewer than 222 items the 4 warps per item are fewer than three quarters of the shares' 1184 workers:
+    // long items then go faster as shares)
+    if (pl.rows_per_item == 8 && 4 * pl.items >= 3 * kPlanSms * 2 && pl.items <= 3 * kPlanSms &&
+        pl.tiles_per_item >= 2 * kWarpsGroup) {
         pl.group_g = kWarpsGroup;
         pl.whole = false;  // (from 8 tiles on, four warps with a merge in shared memory beat one warp alone)
     }

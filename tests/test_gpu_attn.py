@@ -69,6 +69,19 @@ def test_configs_full_size(config_id):
     print(f"config {config_id}: max err / rms = {worst:.2e}")
 
 
+@pytest.mark.parametrize("config_id,overrides", [
+    (2, {}),                                        # 320 items of 36 tiles: four warps of one block per item
+    (4, {}),                                        # 256 items, D = 128
+    (1, dict(B=28, K=5, H=4, H_kv=4, L=300)),       # 224 items of 10 tiles: the smallest call that takes this shape
+    (1, dict(B=37, K=8, H=6, H_kv=6, L=700)),       # 444 items: the largest
+])
+def test_items_merged_inside_a_block_ragged(config_id, overrides):
+    """Few long items of 8 rows: an item's four warps merge in shared memory; with ragged prefix lengths some of
+    a short stream's four shares lie past its last visible key and contribute nothing."""
+    cfg = wl.config(config_id, **overrides)
+    _check(cfg, 700 + config_id + len(overrides), ragged=True, poison_tail=bool(overrides))
+
+
 @pytest.mark.parametrize("L", wl.XL_PREFIX_SWEEP)
 def test_xl_prefix_sweep(L):
     _check(wl.config(2, L=L), wl.seed_for(2, L))
