@@ -796,8 +796,9 @@ __global__ void __launch_bounds__(NT) tree_rows_kernel(const TreeParams P)
 // the spatial sampling pool): one block per (sequence, pool row) draws one token by inverse CDF in
 // ascending id, with the same scan and search as the correction token above.
 template <int NT, int VPT>
-__global__ void __launch_bounds__(NT) pool_sample_kernel(const float *pool_q, const float *u, int32_t *row_token,
-                                                         int V, int v_begin, int n, int vec_ok)
+__global__ void __launch_bounds__(NT) pool_sample_kernel(const float *pool_q, const float *u, const int32_t *node_q,
+                                                         int32_t *node_token, int NQ, int N, int V, int v_begin, int n,
+                                                         int vec_ok, int32_t *dev_status)
 {
     __shared__ RowShared<NT, VPT> sh;
     const int tid = threadIdx.x;
@@ -818,28 +819,21 @@ __global__ void __launch_bounds__(NT) pool_sample_kernel(const float *pool_q, co
     const float total = row_mass<NT, VPT>(x, sj, incl, sh);
     int tok = -1;
     if (total > 0.f) tok = row_search<NT, VPT>(x, sj, incl, ur * total, sh);
-    if (tid == 0) row_token[blockIdx.x] = tok >= 0 ? v_begin + tok : -1;
-}
-
-// node_token[b][node] = the draw of the pool row the node's candidate comes from (node 0, the root, gets 0).
-__global__ void pool_scatter_kernel(const int32_t *row_token, const int32_t *node_q, int32_t *node_token, int B, int NQ,
-                                    int N, int32_t *dev_status)
-{
-    hawk::allow_dependent_launch();
-    hawk::grid_dependency_wait();
-    const int idx = blockIdx.x * blockDim.x + threadIdx.x;
-    if (idx >= B * N) return;
-    const int b = idx / N, node = idx - b * N;
-    int tok = 0;
-    if (node > 0) {
-        int r = node_q[node];
-        if (r < 0 || r >= NQ) {
-            if (dev_status) atomicOr(dev_status, HAWK_DEV_BAD_TREE);
-            r = max(0, min(r, NQ - 1));
+    // every tree node that stands for this pool row carries the draw (the root, node 0, carries 0); a node_q
+    // entry outside [0, NQ) is served by the first or the last row and flagged
+    const int b = blockIdx.x / NQ, r = blockIdx.x - b * NQ;
+    const int token = tok >= 0 ? v_begin + tok : -1;
+    int bad = 0;
+    for (int node = tid; node < N; node += NT) {
+        if (node == 0) {
+            if (r == 0) node_token[b * N] = 0;
+            continue;
         }
-        tok = row_token[b * NQ + r];
+        const int want = node_q[node];
+        bad |= (want < 0 || want >= NQ) ? 1 : 0;
+        if (max(0, min(want, NQ - 1)) == r) node_token[b * N + node] = token;
     }
-    node_token[idx] = tok;
+    if (bad && dev_status) atomicOr(dev_status, HAWK_DEV_BAD_TREE);
 }
 
 // For calls with more rows than SMs: marks every verdict "unknown" and writes each node's parent (the
@@ -1173,25 +1167,21 @@ extern "C" hawk_status hawk_pool_sample(const float *pool_q, const float *u, con
     if (!hawk_host::aligned16(workspace)) return HAWK_ERR_ALIGN;
     if (!hawk_host::is_sm100(nullptr)) return HAWK_ERR_UNSUPPORTED;
     cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
-    int32_t *row_token = static_cast<int32_t *>(workspace);
     const int vec_ok = (V % 4 == 0 && v_begin % 4 == 0) ? 1 : 0;
     const int grid = B * NQ;
     cudaError_t err;
     if (n <= 4096)
-        err = hawk_host::launch_dependent(pool_sample_kernel<256, 4>, dim3(grid), dim3(256), 0, st, pool_q, u, row_token, V,
-                                          v_begin, n, vec_ok);
+        err = hawk_host::launch_dependent(pool_sample_kernel<256, 4>, dim3(grid), dim3(256), 0, st, pool_q, u, node_q,
+                                          node_token, NQ, N, V, v_begin, n, vec_ok, dev_status);
     else if (n <= 8192)
-        err = hawk_host::launch_dependent(pool_sample_kernel<512, 4>, dim3(grid), dim3(512), 0, st, pool_q, u, row_token, V,
-                                          v_begin, n, vec_ok);
+        err = hawk_host::launch_dependent(pool_sample_kernel<512, 4>, dim3(grid), dim3(512), 0, st, pool_q, u, node_q,
+                                          node_token, NQ, N, V, v_begin, n, vec_ok, dev_status);
     else if (n <= 16384)
-        err = hawk_host::launch_dependent(pool_sample_kernel<1024, 4>, dim3(grid), dim3(1024), 0, st, pool_q, u, row_token,
-                                          V, v_begin, n, vec_ok);
+        err = hawk_host::launch_dependent(pool_sample_kernel<1024, 4>, dim3(grid), dim3(1024), 0, st, pool_q, u, node_q,
+                                          node_token, NQ, N, V, v_begin, n, vec_ok, dev_status);
     else
-        err = hawk_host::launch_dependent(pool_sample_kernel<1024, 8>, dim3(grid), dim3(1024), 0, st, pool_q, u, row_token,
-                                          V, v_begin, n, vec_ok);
-    if (err != cudaSuccess) return HAWK_ERR_CUDA;
-    err = hawk_host::launch_dependent(pool_scatter_kernel, dim3((B * N + 255) / 256), dim3(256), 0, st,
-                                      static_cast<const int32_t *>(row_token), node_q, node_token, B, NQ, N, dev_status);
+        err = hawk_host::launch_dependent(pool_sample_kernel<1024, 8>, dim3(grid), dim3(1024), 0, st, pool_q, u, node_q,
+                                          node_token, NQ, N, V, v_begin, n, vec_ok, dev_status);
     return err == cudaSuccess ? HAWK_OK : HAWK_ERR_CUDA;
 }
 
