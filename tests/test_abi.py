@@ -57,8 +57,12 @@ def test_workspace_queries(lib):
     # invalid shapes report 0; a launch that cuts items needs two 16-row fp32 partial slots per share
     assert lib.hawk_verify_attn_workspace_bytes(0, 4, 16, 16, 64, 128) == 0
     assert lib.hawk_verify_attn_workspace_bytes(2, 4, 16, 16, 96, 128) == 0
-    need = lib.hawk_verify_attn_workspace_bytes(16, 5, 20, 20, 64, 1144)
-    assert need > 0 and need % (2 * 8 * 66 * 4) == 0          # K = 5 rows round up to 8 per item
+    need = lib.hawk_verify_attn_workspace_bytes(64, 6, 24, 24, 64, 1144)   # 1536 items cut into equal shares
+    assert need > 0 and need % (2 * 8 * 66 * 4) == 0          # K = 6 rows round up to 8 per item
+    # 320 long items of 8 rows: the four warps of a block share an item and merge in shared memory
+    assert lib.hawk_verify_attn_workspace_bytes(16, 5, 20, 20, 64, 1144) == 0
+    # the same items with 24 tree rows each are cut into shares again
+    assert lib.hawk_verify_attn_workspace_bytes(16, 22, 20, 20, 64, 1144) > 0
     # one tile per item and one share per tile: nothing is cut, no workspace
     assert lib.hawk_verify_attn_workspace_bytes(2, 1, 1, 1, 64, 0) == 0
     assert lib.hawk_cfg_accept_workspace_bytes(8, 5, 16384) >= 8 * 5 * 4
