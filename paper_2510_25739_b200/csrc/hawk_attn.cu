@@ -22,6 +22,8 @@
 //     small second kernel merges the partials of every item that was cut.
 #include <math_constants.h>
 
+#include <atomic>
+
 #include "hawk_common.cuh"
 
 namespace {
@@ -845,12 +847,16 @@ cudaError_t launch_attn_shape(const CUtensorMap &map_k, const CUtensorMap &map_v
                               cudaStream_t st)
 {
     constexpr size_t smem = AttnCfg<D>::smem_bytes(WARPS, STAGES);
-    static bool attr_done = false;
-    if (!attr_done) {
-        const cudaError_t e = cudaFuncSetAttribute(attn_kernel<D, NQT, WARPS, STAGES>,
-                                                   cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+    int device = 0;
+    cudaError_t e = cudaGetDevice(&device);
+    if (e != cudaSuccess) return e;
+    if (device < 0 || device >= 64) return cudaErrorInvalidDevice;
+    static std::atomic<unsigned long long> attr_done{0};  // one bit per device: the limit is a per-device attribute of the function
+    if (!((attr_done.load(std::memory_order_relaxed) >> device) & 1ull)) {
+        e = cudaFuncSetAttribute(attn_kernel<D, NQT, WARPS, STAGES>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 static_cast<int>(smem));
         if (e != cudaSuccess) return e;
-        attr_done = true;
+        attr_done.fetch_or(1ull << device, std::memory_order_relaxed);
     }
     return hawk_host::launch_dependent(attn_kernel<D, NQT, WARPS, STAGES>, dim3(grid), dim3(WARPS * 32), smem, st, map_k,
                                        map_v, P);

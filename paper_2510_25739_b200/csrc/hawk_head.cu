@@ -18,6 +18,8 @@
 // accumulators of a pair (subtract, fused multiply-add, divide: the arithmetic of the accept kernels)
 // and writes ONE row of guided logits, so the logits cross HBM half as often on the way out and half
 // as often on the way into the accept stage.
+#include <atomic>
+
 #include "hawk_common.cuh"
 
 namespace {
@@ -511,14 +513,14 @@ hawk_status head_proj_impl(const void *x, const void *w, float *logits, int M, i
     const size_t smem_req = smem_bytes < 120 * 1024 ? 120 * 1024 : smem_bytes;
     int device = 0;
     if (cudaGetDevice(&device) != cudaSuccess || device < 0 || device >= 64) return HAWK_ERR_CUDA;
-    static unsigned long long attr_done = 0;  // per device: the dynamic shared memory limit is a per-device attribute
-    if (!((attr_done >> device) & 1ull)) {
+    static std::atomic<unsigned long long> attr_done{0};  // per device: the dynamic shared memory limit is a per-device attribute
+    if (!((attr_done.load(std::memory_order_relaxed) >> device) & 1ull)) {
         if (cudaFuncSetAttribute(head_proj_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) !=
                 cudaSuccess ||
             cudaFuncSetAttribute(head_proj_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) !=
                 cudaSuccess)
             return HAWK_ERR_CUDA;
-        attr_done |= 1ull << device;
+        attr_done.fetch_or(1ull << device, std::memory_order_relaxed);
     }
     // few tiles and a long hidden dimension (a narrow valid range of a wide model): split every tile's k-blocks
     // over two blocks so that twice as many SMs stream the weights; plain logits only (the guidance combine
