@@ -51,6 +51,7 @@ struct HeadParams {
 // the tile's token columns 16 at a time; lanes of a warp hold consecutive ids, so every store
 // instruction writes 128 contiguous bytes of one logits row.
 // Warps that share a lane quarter split the 16-column chunks among themselves (chunk0, chunk_step).
+template <bool KSPLIT = false>
 __device__ __forceinline__ void epilogue_store(const HeadParams &P, uint32_t taddr, int tn, int v, bool v_ok,
                                                int chunk0 = 0, int chunk_step = 1)
 {
@@ -66,8 +67,8 @@ __device__ __forceinline__ void epilogue_store(const HeadParams &P, uint32_t tad
                     const int n = n0 + c + j;
                     if (n < P.M) {
                         float *dst = &P.logits[static_cast<size_t>(n) * P.V + v];
-                        if (P.ksplit == 1) *dst = __uint_as_float(r[j]);
-                        else atomicAdd(dst, __uint_as_float(r[j]));  // two addends onto zero: the order cannot matter
+                        if constexpr (KSPLIT) atomicAdd(dst, __uint_as_float(r[j]));  // two addends onto zero: any order
+                        else *dst = __uint_as_float(r[j]);
                     }
                 }
             }
@@ -94,6 +95,8 @@ __device__ __forceinline__ void epilogue_store(const HeadParams &P, uint32_t tad
     }
 }
 
+// KSPLIT: a unit of work is half of a tile's k-blocks and the halves add their results (see head_proj_impl).
+template <bool KSPLIT>
 __global__ void __launch_bounds__(kHeadThreads, 1) head_proj_kernel(const __grid_constant__ CUtensorMap map_w,
                                                                     const __grid_constant__ CUtensorMap map_x,
                                                                     const HeadParams P)
@@ -111,8 +114,9 @@ __global__ void __launch_bounds__(kHeadThreads, 1) head_proj_kernel(const __grid
     hawk::allow_dependent_launch();
     const int kblocks = P.hidden / kBK;
     // a unit of work is a tile, or (ksplit == 2) one half of a tile's k-blocks; the halves add their results
-    const int total_tiles = P.tiles_m * P.tiles_n * P.ksplit;
-    const int kb_half = (kblocks + P.ksplit - 1) / P.ksplit;
+    constexpr int kSplit = KSPLIT ? 2 : 1;
+    const int total_tiles = P.tiles_m * P.tiles_n * kSplit;
+    const int kb_half = (kblocks + kSplit - 1) / kSplit;
 
     if (tid == 0) {
         for (int i = 0; i < P.stages; ++i) {
@@ -147,7 +151,7 @@ __global__ void __launch_bounds__(kHeadThreads, 1) head_proj_kernel(const __grid
             bool ok = true;
             long long issued = 0;
             for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
-                const int part = tile % P.ksplit, t2 = tile / P.ksplit;
+                const int part = tile % kSplit, t2 = tile / kSplit;
                 const int tn = t2 % P.tiles_n, tm = t2 / P.tiles_n;
                 const int row_w = P.v_begin + tm * kBM, row_x = tn * P.BN;
                 const int kb0 = part * kb_half, kb1 = min(kblocks, kb0 + kb_half);
@@ -192,7 +196,7 @@ __global__ void __launch_bounds__(kHeadThreads, 1) head_proj_kernel(const __grid
                 if (!ok) break;
                 tcgen05_fence_after();
                 const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(ab * P.BN);
-                const int part = tile % P.ksplit;
+                const int part = tile % kSplit;
                 const int kb0 = part * kb_half, kb1 = min(kblocks, kb0 + kb_half);
                 for (int kb = kb0; kb < kb1; ++kb) {
                     ok = mbar_wait(&full_bar[st], ph, abort_flag);
@@ -227,7 +231,7 @@ __global__ void __launch_bounds__(kHeadThreads, 1) head_proj_kernel(const __grid
         bool ok = true;
         int it = 0;
         for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++it) {
-            const int t2 = tile / P.ksplit;
+            const int t2 = tile / kSplit;
             const int tn = t2 % P.tiles_n, tm = t2 / P.tiles_n;
             const int ab = it & 1;
             const uint32_t acc_ph = (it >> 1) & 1;
@@ -237,7 +241,7 @@ __global__ void __launch_bounds__(kHeadThreads, 1) head_proj_kernel(const __grid
             const int v = P.v_begin + tm * kBM + lane_base + lane;  // this thread's token id
             const bool v_ok = v < P.v_end;
             const uint32_t taddr = tmem_base + (static_cast<uint32_t>(lane_base) << 16) + static_cast<uint32_t>(ab * P.BN);
-            epilogue_store(P, taddr, tn, v, v_ok);
+            epilogue_store<KSPLIT>(P, taddr, tn, v, v_ok);
             tcgen05_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(&acc_empty[ab]);
@@ -515,7 +519,9 @@ hawk_status head_proj_impl(const void *x, const void *w, float *logits, int M, i
     if (cudaGetDevice(&device) != cudaSuccess || device < 0 || device >= 64) return HAWK_ERR_CUDA;
     static std::atomic<unsigned long long> attr_done{0};  // per device: the dynamic shared memory limit is a per-device attribute
     if (!((attr_done.load(std::memory_order_relaxed) >> device) & 1ull)) {
-        if (cudaFuncSetAttribute(head_proj_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) !=
+        if (cudaFuncSetAttribute(head_proj_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) !=
+                cudaSuccess ||
+            cudaFuncSetAttribute(head_proj_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) !=
                 cudaSuccess ||
             cudaFuncSetAttribute(head_proj_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) !=
                 cudaSuccess)
@@ -557,8 +563,9 @@ hawk_status head_proj_impl(const void *x, const void *w, float *logits, int M, i
                                           reinterpret_cast<cudaStream_t>(stream), map_w, map_x, P);
     } else {
         const int grid = total_tiles < sm_count ? total_tiles : sm_count;
-        err = hawk_host::launch_dependent(head_proj_kernel, dim3(grid), dim3(kHeadThreads), smem_req,
-                                          reinterpret_cast<cudaStream_t>(stream), map_w, map_x, P);
+        err = hawk_host::launch_dependent(P.ksplit > 1 ? head_proj_kernel<true> : head_proj_kernel<false>, dim3(grid),
+                                          dim3(kHeadThreads), smem_req, reinterpret_cast<cudaStream_t>(stream), map_w,
+                                          map_x, P);
     }
     return err == cudaSuccess ? HAWK_OK : HAWK_ERR_CUDA;
 }
