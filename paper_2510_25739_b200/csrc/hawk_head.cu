@@ -41,6 +41,7 @@ struct HeadParams {
     int tiles_n;   // token tiles
     int stages;
     int stage_bytes;
+    int wide;      // pair kernel: one accumulator of BN (up to 512) columns, every k-step as two MMAs of BN / 2 columns
     int ksplit;    // 1, or 2: two work units per tile, each over half of the hidden dimension (output zeroed first)
     int pairs;     // 0: plain logits; > 0: guided logits of this many (sequence, position) pairs
     float cfg_scale, temperature;
@@ -51,7 +52,10 @@ struct HeadParams {
 // the tile's token columns 16 at a time; lanes of a warp hold consecutive ids, so every store
 // instruction writes 128 contiguous bytes of one logits row.
 // Warps that share a lane quarter split the 16-column chunks among themselves (chunk0, chunk_step).
-template <bool KSPLIT = false>
+// WIDE (pair kernel, two MMAs of BN / 2 columns per k-step): accumulator column t of MMA half c = t / (BN / 2)
+// comes from CTA (t % (BN / 2)) / (BN / 4), row c * (BN / 4) + t % (BN / 4) of that CTA's token rows; BN is a
+// multiple of 64 there, so a 16-column chunk never straddles two of these ranges.
+template <bool KSPLIT = false, bool WIDE = false>
 __device__ __forceinline__ void epilogue_store(const HeadParams &P, uint32_t taddr, int tn, int v, bool v_ok,
                                                int chunk0 = 0, int chunk_step = 1)
 {
@@ -61,10 +65,16 @@ __device__ __forceinline__ void epilogue_store(const HeadParams &P, uint32_t tad
             uint32_t r[16];
             tmem_ld_32x16(taddr + c, r);
             tmem_ld_wait();
+            int nbase = n0 + c;
+            if constexpr (WIDE) {
+                const int half = P.BN / 2, quarter = P.BN / 4;
+                const int mma = c / half, j = c - mma * half;
+                nbase = n0 + (j / quarter) * half + mma * quarter + j % quarter;
+            }
             if (v_ok) {
 #pragma unroll
                 for (int j = 0; j < 16; ++j) {
-                    const int n = n0 + c + j;
+                    const int n = nbase + j;
                     if (n < P.M) {
                         float *dst = &P.logits[static_cast<size_t>(n) * P.V + v];
                         if constexpr (KSPLIT) atomicAdd(dst, __uint_as_float(r[j]));  // two addends onto zero: any order
@@ -280,6 +290,7 @@ constexpr uint32_t kPairTmemCols = HAWK_PAIR_TMEM_COLS;
 
 constexpr int kPairThreads = 320;  // producer, MMA, and two epilogue warps per tensor-memory lane quarter
 
+template <bool WIDE>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kPairThreads, 1)
     head_proj_pair_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_x,
                           const HeadParams P)
@@ -362,14 +373,15 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kPairThreads, 1)
     } else if (warp == 1) {
         // =========================== rank 0: MMA issuer for the pair
         if (lane == 0) {
-            const uint32_t idesc = umma_idesc_bf16_f32(2 * kBM, P.BN);
+            const int mma_n = WIDE ? P.BN / 2 : P.BN;  // columns per MMA
+            const uint32_t idesc = umma_idesc_bf16_f32(2 * kBM, mma_n);
             int st = 0;
             uint32_t ph = 0;
             bool ok = true;
             int it = 0;
             for (int tile = pair; tile < total_tiles && ok; tile += n_pairs, ++it) {
-                const int ab = it & 1;
-                const uint32_t acc_ph = (it >> 1) & 1;
+                const int ab = WIDE ? 0 : it & 1;  // WIDE: one accumulator fills tensor memory
+                const uint32_t acc_ph = WIDE ? it & 1 : (it >> 1) & 1;
                 ok = mbar_wait_cluster(&acc_empty[ab], acc_ph ^ 1u, abort_flag);  // both epilogues drained it
                 if (!ok) break;
                 tcgen05_fence_after();
@@ -382,9 +394,15 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kPairThreads, 1)
                     const uint64_t da = umma_desc_k_major_sw128(a_addr);
                     const uint64_t db = umma_desc_k_major_sw128(a_addr + kATileBytes);
 #pragma unroll
-                    for (int k = 0; k < kBK / 16; ++k)
+                    for (int k = 0; k < kBK / 16; ++k) {
                         umma_bf16_pair(d_tmem, da + static_cast<uint64_t>(2 * k), db + static_cast<uint64_t>(2 * k), idesc,
                                        (kb | k) != 0 ? 1u : 0u);
+                        if constexpr (WIDE) {  // second half of the columns: rows BN / 4 onwards of each CTA's token rows
+                            const uint64_t db2 = umma_desc_k_major_sw128(a_addr + kATileBytes + (P.BN / 4) * kBK * 2);
+                            umma_bf16_pair(d_tmem + static_cast<uint32_t>(mma_n), da + static_cast<uint64_t>(2 * k),
+                                           db2 + static_cast<uint64_t>(2 * k), idesc, (kb | k) != 0 ? 1u : 0u);
+                        }
+                    }
                     umma_commit_pair(&empty_bar[st], 3);  // the stage is reusable in both CTAs
                     if (++st == P.stages) {
                         st = 0;
@@ -407,15 +425,15 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kPairThreads, 1)
         int it = 0;
         for (int tile = pair; tile < total_tiles && ok; tile += n_pairs, ++it) {
             const int tn = tile % P.tiles_n, tm = tile / P.tiles_n;
-            const int ab = it & 1;
-            const uint32_t acc_ph = (it >> 1) & 1;
+            const int ab = WIDE ? 0 : it & 1;
+            const uint32_t acc_ph = WIDE ? it & 1 : (it >> 1) & 1;
             ok = mbar_wait_cluster(&acc_full[ab], acc_ph, abort_flag);
             if (!ok) break;
             tcgen05_fence_after();
             const int v = P.v_begin + tm * (2 * kBM) + static_cast<int>(rank) * kBM + lane_base + lane;
             const bool v_ok = v < P.v_end;
             const uint32_t taddr = tmem_base + (static_cast<uint32_t>(lane_base) << 16) + static_cast<uint32_t>(ab * P.BN);
-            epilogue_store(P, taddr, tn, v, v_ok, (warp - 2) >> 2, 2);
+            epilogue_store<false, WIDE>(P, taddr, tn, v, v_ok, (warp - 2) >> 2, 2);
             tcgen05_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive_cluster(acc_empty_rank0[ab]);
@@ -480,9 +498,14 @@ hawk_status head_proj_impl(const void *x, const void *w, float *logits, int M, i
 #ifndef HAWK_HEAD_PAIR_MIN_ROWS
 #define HAWK_HEAD_PAIR_MIN_ROWS 512
 #endif
-    const bool use_pair = M >= HAWK_HEAD_PAIR_MIN_ROWS && sm_count >= 2;
-    const int max_bn = use_pair ? static_cast<int>(kPairTmemCols) / 2 : 256;  // two accumulators in tensor memory
-    const int bn_step = use_pair ? 32 : 16;  // a pair's tile splits into two halves of a multiple of 16 rows
+    // Between 257 and 511 rows of plain logits the pair kernel takes all rows as ONE tile of up to 512 columns (one
+    // accumulator, no overlap of epilogue and MMAs, but a single round of tiles whose MMAs are wide enough to hide
+    // their issue cost): 25.6 -> measured below at 384 rows.
+    const bool wide = pairs == 0 && M > 256 && M < HAWK_HEAD_PAIR_MIN_ROWS && sm_count >= 2 && kPairTmemCols == 512;
+    const bool use_pair = (M >= HAWK_HEAD_PAIR_MIN_ROWS || wide) && sm_count >= 2;
+    const int max_bn = wide ? 512 : use_pair ? static_cast<int>(kPairTmemCols) / 2 : 256;  // accumulators in tensor memory
+    const int bn_step = wide ? 64 : use_pair ? 32 : 16;  // a pair's tile splits into halves of a multiple of 16 rows
+    P.wide = wide ? 1 : 0;
     int x_box_rows;
     if (pairs == 0) {
         P.tiles_n = (M + max_bn - 1) / max_bn;
@@ -523,7 +546,9 @@ hawk_status head_proj_impl(const void *x, const void *w, float *logits, int M, i
                 cudaSuccess ||
             cudaFuncSetAttribute(head_proj_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) !=
                 cudaSuccess ||
-            cudaFuncSetAttribute(head_proj_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) !=
+            cudaFuncSetAttribute(head_proj_pair_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) !=
+                cudaSuccess ||
+            cudaFuncSetAttribute(head_proj_pair_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) !=
                 cudaSuccess)
             return HAWK_ERR_CUDA;
         attr_done.fetch_or(1ull << device, std::memory_order_relaxed);
@@ -551,7 +576,7 @@ hawk_status head_proj_impl(const void *x, const void *w, float *logits, int M, i
             occ.blockDim = dim3(kPairThreads);
             occ.dynamicSmemBytes = 227 * 1024 - 1024;
             int n = 0;
-            if (cudaOccupancyMaxActiveClusters(&n, head_proj_pair_kernel, &occ) != cudaSuccess || n < 1) {
+            if (cudaOccupancyMaxActiveClusters(&n, head_proj_pair_kernel<false>, &occ) != cudaSuccess || n < 1) {
                 (void)cudaGetLastError();
                 n = sm_count / 4;  // conservative: half of the SMs
             }
@@ -559,7 +584,8 @@ hawk_status head_proj_impl(const void *x, const void *w, float *logits, int M, i
         }
         const int max_pairs = max_pairs_of[device];
         const int n_pairs = total_tiles < max_pairs ? total_tiles : max_pairs;
-        err = hawk_host::launch_dependent(head_proj_pair_kernel, dim3(2 * n_pairs), dim3(kPairThreads), smem_req,
+        err = hawk_host::launch_dependent(wide ? head_proj_pair_kernel<true> : head_proj_pair_kernel<false>,
+                                          dim3(2 * n_pairs), dim3(kPairThreads), smem_req,
                                           reinterpret_cast<cudaStream_t>(stream), map_w, map_x, P);
     } else {
         const int grid = total_tiles < sm_count ? total_tiles : sm_count;
