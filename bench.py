@@ -47,8 +47,8 @@ L2_BYTES = 126 * 1024 * 1024
 # current kernels exists for that workload.
 NOMINAL_HBM_GBS = 7700.0       # HBM3e figure of the HGX B200 data sheet
 NOMINAL_BF16_TFLOPS = 2250.0   # dense bf16
-ATTN_TRAFFIC_BYTES = {2: 94_549_000 + 3_696_000,                 # attention kernel read + write (no merge kernel at this shape)
-                      5: 679_406_000 + 5_353_000 + 4_757_000}   # attention read + write, merge kernel read
+ATTN_TRAFFIC_BYTES = {2: 94_548_000 + 5_019_000,                 # attention kernel read + write (no merge kernel at this shape)
+                      5: 679_447_000 + 4_913_000 + 4_756_000}   # attention read + write, merge kernel read
 
 
 def measured_peaks():
