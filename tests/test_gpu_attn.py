@@ -74,6 +74,8 @@ def test_configs_full_size(config_id):
     (4, {}),                                        # 256 items, D = 128
     (1, dict(B=28, K=5, H=4, H_kv=4, L=300)),       # 224 items of 10 tiles: the smallest call that takes this shape
     (1, dict(B=37, K=8, H=6, H_kv=6, L=700)),       # 444 items: the largest
+    (1, dict(B=19, K=3, H=12, H_kv=6, D=128, L=211)),  # 228 items, two query heads per kv head (6 of 8 rows used)
+    (1, dict(B=63, K=1, H=6, H_kv=3, D=128, L=628)),   # one draft, grouped-query heads
 ])
 def test_items_merged_inside_a_block_ragged(config_id, overrides):
     """Few long items of 8 rows: an item's four warps merge in shared memory; with ragged prefix lengths some of

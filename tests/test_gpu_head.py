@@ -45,6 +45,7 @@ SMALL = [
     (300, 256, 384, 0, 384),       # 257..511 rows: CTA pairs, one tile of all rows (two MMAs of half the columns)
     (384, 192, 700, 3, 697),       # the same at 384 rows with ragged 256-id tiles
     (500, 128, 512, 0, 512),       # ... and at 500 rows (512 accumulator columns)
+    (333, 1856, 2475, 4, 2467),    # ... with 29 k-blocks and a ragged range
     (17, 1024, 2048, 0, 2048),     # more k-blocks than pipeline stages; few tiles: each split over two blocks along hidden
     (48, 1088, 1000, 4, 996),      # split along hidden with an odd number of k-blocks (17), ragged range
     (600, 320, 700, 1, 699),       # three token tiles, ragged both ways (from 512 rows on: the CTA-pair kernel)
