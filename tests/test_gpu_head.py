@@ -52,6 +52,8 @@ SMALL = [
     (512, 128, 256, 0, 256),       # CTA pairs: one tile of 256 ids x 256 rows per pair, two token tiles
     (1000, 192, 900, 3, 897),      # CTA pairs: ragged 256-id tiles, four token tiles of 256 rows (the last ragged)
     (513, 1024, 512, 0, 512),      # CTA pairs: three token tiles of 192 rows, more k-blocks than stages
+    (1024, 128, 5120, 0, 5120),    # CTA pairs: 80 tiles on 74 pairs, a second, partly empty round
+    (1000, 192, 5000, 7, 4990),    # ... ragged in both directions
 ]
 
 

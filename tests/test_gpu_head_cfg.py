@@ -44,6 +44,8 @@ CASES = [
     (3, 22, 1024, 2048, 0, 2048, 3.0, 1.0),      # tree-shaped rows, more k-blocks than stages
     (32, 8, 256, 1024, 0, 1024, 3.0, 1.0),       # 256 pairs = 512 rows: the CTA-pair kernel, two tiles of 128 pairs
     (40, 9, 128, 700, 5, 690, 7.5, 0.9),         # 360 pairs: CTA pairs, three ragged tiles
+    (64, 8, 128, 5120, 0, 5120, 3.0, 1.0),       # 512 pairs, 80 tiles on 74 CTA pairs: two rounds
+    (50, 10, 64, 5000, 3, 4995, 7.5, 0.8),       # 500 pairs, the same ragged
 ]
 
 
