@@ -165,3 +165,82 @@ def test_attn_tree_argument_checks(lib):
     assert f(p, p, p, p, p, p, 0, 7, 4, 4, 64, 100, 90, 0.125, None, 0, None, None) == OK
     assert f(p, p, p, p, p, p, 2, 33, 4, 4, 64, 200, 90, 0.125, None, 0, None, None) == E_UNSUP
     assert f(p, p, p, p, p, p, 2, 22, 4, 4, 64, 100, 90, 0.125, None, 0, None, None) == E_SHAPE    # 90 + 22 > 100
+
+
+def test_guided_head_and_accept_argument_checks(lib):
+    p, odd = ctypes.c_void_p(0x1000), ctypes.c_void_p(0x1008)
+    f = lib.hawk_head_proj_cfg
+    c = ctypes.c_float
+
+    def head(x=p, w=p, out=p, B=2, rows=4, hidden=1024, V=16384, vb=0, ve=16384, s=3.0, T=1.0):
+        return f(x, w, out, B, rows, hidden, V, vb, ve, c(s), c(T), None, None)
+
+    assert head(B=0) == OK
+    assert head(B=-1) == E_SHAPE and head(rows=-1) == E_SHAPE
+    assert head(ve=16385) == E_SHAPE
+    assert head(x=None) == E_NULL and head(out=None) == E_NULL
+    assert head(hidden=1000) == E_UNSUP
+    assert head(T=0.0) == E_PARAM and head(T=float("nan")) == E_PARAM and head(s=float("inf")) == E_PARAM
+    assert head(w=odd) == E_ALIGN
+
+    g = lib.hawk_cfg_accept_guided
+
+    def acc(lg=p, q=p, d=p, ua=p, ur=p, B=2, K=4, V=1024, vb=0, ve=1024, k=100, al=p, tok=p, ws=p, wsb=1 << 20):
+        return g(lg, q, d, ua, ur, B, K, V, vb, ve, k, 0, al, tok, None, ws, wsb, None, None)
+
+    assert acc(B=0) == OK
+    assert acc(B=-1) == E_SHAPE
+    assert acc(lg=None) == E_NULL and acc(al=None) == E_NULL
+    assert acc(vb=10, ve=10) == E_SHAPE
+    assert acc(K=17) == E_UNSUP
+    assert acc(q=odd) == E_ALIGN
+    assert acc(ws=None) == E_WS
+
+    t = lib.hawk_tree_accept_guided
+
+    def tree(lg=p, q=p, tokn=p, nq=p, cb=p, ua=p, ur=p, B=2, N=7, NQ=4, V=1024, vb=0, ve=1024, k=100, md=3, al=p, tok=p,
+             path=p, ws=p, wsb=1 << 20):
+        return t(lg, q, tokn, nq, cb, ua, ur, B, N, NQ, V, vb, ve, k, md, al, tok, path, ws, wsb, None, None)
+
+    assert tree(B=0) == OK
+    assert tree(N=0) == E_SHAPE and tree(NQ=0) == E_SHAPE and tree(md=-1) == E_SHAPE
+    assert tree(cb=None) == E_NULL
+    assert tree(V=40000, ve=40000) == E_UNSUP
+    assert tree(wsb=8) == E_WS
+
+
+def test_cache_and_pool_argument_checks(lib):
+    p, odd = ctypes.c_void_p(0x1000), ctypes.c_void_p(0x1004)
+    assert lib.hawk_spec_cache_slots(32, 2) == 96 and lib.hawk_spec_cache_slots(48, 3) == 288
+    assert lib.hawk_spec_cache_slots(0, 2) == 0 and lib.hawk_spec_cache_slots(32, 0) == 0
+    # slots of one column and depth cycle with period `depth`; different depths never share a slot
+    assert lib.hawk_spec_cache_slot(4, 2, 0, 1) == 0 and lib.hawk_spec_cache_slot(4, 2, 4, 1) == 0
+    assert lib.hawk_spec_cache_slot(4, 2, 0, 2) == 1 and lib.hawk_spec_cache_slot(4, 2, 4, 2) == 2
+    assert lib.hawk_spec_cache_slot(4, 2, 8, 2) == 1 and lib.hawk_spec_cache_slot(4, 2, 1, 1) == 3
+    assert lib.hawk_spec_cache_slot(4, 2, -1, 1) == -1 and lib.hawk_spec_cache_slot(4, 2, 0, 3) == -1
+    assert lib.hawk_spec_cache_clear(None, 2, 4, 2, None) == E_NULL
+    assert lib.hawk_spec_cache_clear(p, 0, 4, 2, None) == OK
+    assert lib.hawk_spec_cache_clear(p, 2, 0, 2, None) == E_SHAPE
+    put = lib.hawk_spec_cache_put
+    assert put(p, p, p, p, 0, 4, 2, 64, None) == OK
+    assert put(None, p, p, p, 2, 4, 2, 64, None) == E_NULL
+    assert put(p, p, p, p, 2, 4, 2, 0, None) == E_SHAPE
+    assert put(p, p, p, p, 2, 4, 9, 64, None) == E_UNSUP
+    build_ = lib.hawk_pool_build
+    assert build_(p, p, p, p, p, None, 0, 3, 4, 2, 64, None) == OK
+    assert build_(p, p, p, p, p, None, 2, 0, 4, 2, 64, None) == OK
+    assert build_(p, p, p, p, None, None, 2, 3, 4, 2, 64, None) == E_NULL
+    assert build_(p, p, p, p, p, None, 2, 3, 0, 2, 64, None) == E_SHAPE
+    assert build_(p, p, p, p, p, None, 2, 3, 4, 9, 64, None) == E_UNSUP
+    assert lib.hawk_pool_sample_workspace_bytes(2, 9) == 72 and lib.hawk_pool_sample_workspace_bytes(0, 9) == 0
+    samp = lib.hawk_pool_sample
+
+    def sample(pq=p, u=p, nq=p, out=p, B=2, NQ=9, N=22, V=1024, vb=0, ve=1024, ws=p, wsb=1 << 10):
+        return samp(pq, u, nq, out, B, NQ, N, V, vb, ve, ws, wsb, None, None)
+
+    assert sample(B=0) == OK
+    assert sample(B=-1) == E_SHAPE and sample(NQ=0) == E_SHAPE and sample(vb=5, ve=5) == E_SHAPE
+    assert sample(out=None) == E_NULL
+    assert sample(V=40000, ve=40000) == E_UNSUP
+    assert sample(pq=odd) == E_ALIGN
+    assert sample(wsb=8) == E_WS
