@@ -84,12 +84,20 @@ __device__ __forceinline__ void epilogue_store(const HeadParams &P, uint32_t tad
             }
         }
     } else {
-        const int half = P.BN / 2;  // a multiple of 16
+        const int half = P.BN / 2;  // pairs per tile, a multiple of 16
         const bool unit_T = P.temperature == 1.0f;
         for (int c = 16 * chunk0; c < half; c += 16 * chunk_step) {
             uint32_t rc[16], ru[16];
-            tmem_ld_32x16(taddr + c, rc);
-            tmem_ld_32x16(taddr + half + c, ru);
+            // columns of pairs c .. c + 15: conditional rows, then unconditional rows; WIDE: MMA half m = c / (BN / 4)
+            // holds the conditional rows of its pairs in its first BN / 4 columns, the unconditional ones in the rest
+            int col_c = c, col_u = half + c;
+            if constexpr (WIDE) {
+                const int quarter = P.BN / 4, m = c / quarter, jj = c - m * quarter;
+                col_c = m * half + jj;
+                col_u = col_c + quarter;
+            }
+            tmem_ld_32x16(taddr + col_c, rc);
+            tmem_ld_32x16(taddr + col_u, ru);
             tmem_ld_wait();
             if (v_ok) {
 #pragma unroll
@@ -498,10 +506,10 @@ hawk_status head_proj_impl(const void *x, const void *w, float *logits, int M, i
 #ifndef HAWK_HEAD_PAIR_MIN_ROWS
 #define HAWK_HEAD_PAIR_MIN_ROWS 512
 #endif
-    // Between 257 and 511 rows of plain logits the pair kernel takes all rows as ONE tile of up to 512 columns (one
+    // Between 257 and 511 token rows the pair kernel takes all rows as ONE tile of up to 512 columns (one
     // accumulator, no overlap of epilogue and MMAs, but a single round of tiles whose MMAs are wide enough to hide
     // their issue cost): 25.6 -> measured below at 384 rows.
-    const bool wide = pairs == 0 && M > 256 && M < HAWK_HEAD_PAIR_MIN_ROWS && sm_count >= 2 && kPairTmemCols == 512;
+    const bool wide = M > 256 && M < HAWK_HEAD_PAIR_MIN_ROWS && sm_count >= 2 && kPairTmemCols == 512;
     const bool use_pair = (M >= HAWK_HEAD_PAIR_MIN_ROWS || wide) && sm_count >= 2;
     const int max_bn = wide ? 512 : use_pair ? static_cast<int>(kPairTmemCols) / 2 : 256;  // accumulators in tensor memory
     const int bn_step = wide ? 64 : use_pair ? 32 : 16;  // a pair's tile splits into halves of a multiple of 16 rows
@@ -512,10 +520,11 @@ hawk_status head_proj_impl(const void *x, const void *w, float *logits, int M, i
         const int per_tile = (M + P.tiles_n - 1) / P.tiles_n;
         P.BN = (per_tile + bn_step - 1) / bn_step * bn_step;
         x_box_rows = use_pair ? P.BN / 2 : P.BN;
-    } else {  // half a tile of conditional rows, half of unconditional ones; each half a multiple of 16
+    } else {  // half a tile of conditional rows, half of unconditional ones; each half a multiple of 16 (32 when wide)
         P.tiles_n = (pairs + max_bn / 2 - 1) / (max_bn / 2);
         const int per_tile = (pairs + P.tiles_n - 1) / P.tiles_n;
-        x_box_rows = (per_tile + 15) / 16 * 16;
+        const int step = wide ? 32 : 16;
+        x_box_rows = (per_tile + step - 1) / step * step;
         P.BN = 2 * x_box_rows;
     }
     const int tile_rows = use_pair ? 2 * kBM : kBM;  // token ids per tile

@@ -42,6 +42,9 @@ CASES = [
     (13, 10, 192, 384, 0, 384, 0.0, 2.0),        # 130 pairs: two token tiles, the second nearly empty
     (30, 10, 320, 700, 1, 699, 3.0, 1.0),        # 300 pairs: three token tiles
     (3, 22, 1024, 2048, 0, 2048, 3.0, 1.0),      # tree-shaped rows, more k-blocks than stages
+    (24, 8, 256, 1024, 0, 1024, 3.0, 1.0),       # 192 pairs = 384 rows: CTA pairs, all rows in one 384-column tile
+    (25, 10, 192, 700, 3, 697, 7.5, 0.9),        # 250 pairs = 500 rows, ragged ids (512 accumulator columns)
+    (13, 10, 128, 512, 0, 512, 3.0, 1.0),        # 130 pairs = 260 rows (320 columns: quarters of 80)
     (32, 8, 256, 1024, 0, 1024, 3.0, 1.0),       # 256 pairs = 512 rows: the CTA-pair kernel, two tiles of 128 pairs
     (40, 9, 128, 700, 5, 690, 7.5, 0.9),         # 360 pairs: CTA pairs, three ragged tiles
     (64, 8, 128, 5120, 0, 5120, 3.0, 1.0),       # 512 pairs, 80 tiles on 74 CTA pairs: two rounds
