@@ -3,16 +3,21 @@
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--config C] [--impl reference]
 
-One "step" is one pass of the whole verify path over one batch of synthetic inputs shaped like
-workload C (default 2: LlamaGen-XL-shaped, KV length 1144).  Rank 0 prints ONE JSON line.
+One "step" is one pass of the whole verify path over one batch of synthetic inputs.  Without --config the
+headline is workload 5 (acceptance stress: the largest of the five that fit one GPU) and the line also carries a
+`per_config` table of all five workloads; --config C measures workload C alone.  Rank 0 prints ONE JSON line.
 
 * value            verified draft positions per second, inputs resident in HBM, whole job (all ranks);
                    each step is a CUDA-graph replay of the three C-ABI calls.
 * e2e              same metric through hawk_verify_step_host: pinned host buffers, host->device
                    copies of the step's inputs and device->host copy of the results inside the
                    timed region.
-* roofline         the dominant kernel (attention), timed with CUDA events inside the timed steps.
-* cpu_baseline     the CPU oracle timed on the host cores on a bounded sample (rank 0, N=1 only).
+* roofline         the kernel with the largest share of the step, timed alone with CUDA events on the bench stream.
+* per_config       for workloads 1..5: step time, positions/s, per-kernel mean / median / min microseconds and each
+                   kernel's fraction of the roofline that bounds it (HBM for attention, accept and the head at few
+                   token rows; tensor for the head at many).
+* cpu_baseline     the CPU oracle timed on the host cores on a bounded sample (rank 0, N=1 only), all cores and once
+                   single-threaded.
 * --impl reference times that same oracle as the reference arm.
 
 Inputs rotate over enough replicas that consecutive steps never find their data in L2.
@@ -38,15 +43,16 @@ if str(ROOT) not in sys.path:
 from paper_2510_25739_b200 import workloads as wl  # noqa: E402
 
 METRIC = "verified draft positions/sec per B200 (verify step)"
+HEADLINE_CONFIG = 5            # the largest of the five workloads that fits one GPU
 UNIT = "positions/s"
 L2_BYTES = 126 * 1024 * 1024
 
 
-# DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) of one hawk_verify_attn call, attention kernel
-# plus merge kernel, from the ncu capture summarised in profiles/; None where no capture of the
-# current kernels exists for that workload.
 NOMINAL_HBM_GBS = 7700.0       # HBM3e figure of the HGX B200 data sheet
 NOMINAL_BF16_TFLOPS = 2250.0   # dense bf16
+# DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) of one hawk_verify_attn call, attention kernel
+# plus merge kernel, from the ncu captures summarised in profiles/ (not measured by this script); an entry is
+# dropped when the attention kernels change and no new capture exists.
 ATTN_TRAFFIC_BYTES = {2: 94_548_000 + 5_019_000,                 # attention kernel read + write (no merge kernel at this shape)
                       5: 679_447_000 + 4_913_000 + 4_756_000}   # attention read + write, merge kernel read
 
@@ -74,10 +80,6 @@ def head_bytes(cfg) -> int:
 
 def head_flops(cfg) -> int:
     return 2 * cfg.M * cfg.hidden * cfg.V_valid
-
-
-def accept_bytes(cfg, q_rows_read: int) -> int:
-    return 2 * cfg.B * cfg.K * cfg.V_valid * 4 + q_rows_read * cfg.V_valid * 4
 
 
 # ------------------------------------------------------------------------------------------ clocks
@@ -239,16 +241,9 @@ def run_accept_guided(cfg, r, hawk):
                            accept_len=r.accept_len2, out_token=r.out_token2, workspace=r.acc_ws, dev_status=r.status)
 
 
-def make_event(torch):
-    try:
-        return torch.cuda.Event(enable_timing=True, external=True), True
-    except TypeError:
-        return torch.cuda.Event(enable_timing=True), False
-
-
 # ------------------------------------------------------------------------------------------ CPU oracle leg
-def oracle_sample(cfg, seed, reps):
-    """Times the CPU oracle (as it stands) on `reps` full steps of the workload; returns positions/s."""
+def oracle_sample(cfg, seed, reps, threads=None):
+    """Times the CPU oracle (as it stands) on `reps` full steps of `cfg`; returns (positions/s, seconds, threads)."""
     import oracle
     a = wl.make_attn_inputs(cfg, seed)
     h = wl.make_head_inputs(cfg, seed)
@@ -256,14 +251,22 @@ def oracle_sample(cfg, seed, reps):
     drafts = wl.draw_drafts(q, seed)
     u = wl.draw_uniforms(cfg, seed)
     oracle.build()
-    t0 = time.perf_counter()
-    for _ in range(reps):
-        oracle.verify_attn(a["q"], a["k_cache"], a["v_cache"], a["prefix_len"], a["sm_scale"])
-        lg = oracle.head_proj(h["x"], h["w"], cfg.v_begin, cfg.v_end, fill=0.0)
-        oracle.cfg_accept(lg.reshape(cfg.S, cfg.K, cfg.V), q, drafts, u["u_accept"], u["u_resample"], cfg.v_begin,
-                          cfg.v_end, cfg.cfg_scale, cfg.temperature, cfg.top_k, diagnostics=False)
-    dt = time.perf_counter() - t0
-    return cfg.B * cfg.K * reps / dt, dt, oracle.threads()
+    all_threads = oracle.threads()
+    if threads is not None:
+        oracle.set_threads(threads)
+    try:
+        t0 = time.perf_counter()
+        for _ in range(reps):
+            oracle.verify_attn(a["q"], a["k_cache"], a["v_cache"], a["prefix_len"], a["sm_scale"])
+            lg = oracle.head_proj(h["x"], h["w"], cfg.v_begin, cfg.v_end, fill=0.0)
+            oracle.cfg_accept(lg.reshape(cfg.S, cfg.K, cfg.V), q, drafts, u["u_accept"], u["u_resample"], cfg.v_begin,
+                              cfg.v_end, cfg.cfg_scale, cfg.temperature, cfg.top_k, diagnostics=False)
+        dt = time.perf_counter() - t0
+        used = oracle.threads()
+    finally:
+        if threads is not None:
+            oracle.set_threads(all_threads)
+    return cfg.B * cfg.K * reps / dt, dt, used
 
 
 def workload_name(cfg, cid):
@@ -273,66 +276,100 @@ def workload_name(cfg, cid):
 
 
 def reference_arm(args, cfg, cid):
+    """The CPU oracle as the reference arm: exactly --steps timed steps after --warmup untimed ones.  A step is the
+    whole workload when that keeps the run within minutes, else the first sequences of it (a bounded sample)."""
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    _, t1, cores = oracle_sample(cfg, wl.seed_for(cid), 1)          # also warms the build and the page cache
-    steps = max(1, min(args.steps, int(120.0 / max(t1, 1e-3))))      # the whole run ends within minutes
-    total = 0.0
-    for _ in range(steps):
-        _, dt, cores = oracle_sample(cfg, wl.seed_for(cid), 1)
-        total += dt
-    value = cfg.B * cfg.K * steps / total
+    seed = wl.seed_for(cid)
+    steps, warmup = max(args.steps, 1), max(args.warmup, 1)
+    probe_B = min(cfg.B, 4)
+    _, t_probe, cores = oracle_sample(replace(cfg, B=probe_B), seed, 1)    # also warms the build and the page cache
+    _, t_probe, cores = oracle_sample(replace(cfg, B=probe_B), seed, 1)
+    per_seq = t_probe / probe_B
+    budget_s = 150.0
+    B_step = int(max(1, min(cfg.B, budget_s / ((steps + warmup) * per_seq))))
+    scfg = replace(cfg, B=B_step)
+    oracle_sample(scfg, seed, warmup)
+    v, total, cores = oracle_sample(scfg, seed, steps)
+    sample = (f"{steps} full steps of the workload" if B_step == cfg.B else
+              f"{steps} steps of the first {B_step} of {cfg.B} sequences of the workload (all {cfg.K} positions, both streams)")
     line = {
-        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": steps,
-        "warmup": 1, "ms_per_step": 1e3 * total / steps, "higher_is_better": True, "scaling": "weak",
+        "impl": "reference", "metric": METRIC, "value": v, "unit": UNIT, "n_gpus": args.gpus, "steps": steps,
+        "warmup": warmup, "ms_per_step": 1e3 * total / steps, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": workload_name(cfg, cid), "note": "CPU oracle, one full step of the workload per step"},
-        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle",
-                         "sample": f"{steps} full steps of the workload"},
-        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "config": {"workload": workload_name(cfg, cid), "note": "CPU oracle; " + sample},
+        "cpu_baseline": {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": v, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
     }
     print(json.dumps(line))
 
 
-# ------------------------------------------------------------------------------------------ main arm
-def main():
-    ap = argparse.ArgumentParser()
-    ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=2000)
-    ap.add_argument("--warmup", type=int, default=20)
-    ap.add_argument("--config", type=int, default=2, help="workload id 1..5 (default 2: LlamaGen-XL-shaped)")
-    ap.add_argument("--impl", default="hawk", choices=["hawk", "reference"])
-    ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--no-e2e", action="store_true")
-    ap.add_argument("--e2e-eager", action="store_true", help="time the end-to-end call eagerly instead of as a graph")
-    ap.add_argument("--graph-events", action="store_true",
-                    help="also record events around the attention call inside the step graphs (perturbs the step)")
-    args = ap.parse_args()
-    cid = args.config
+# ------------------------------------------------------------------------------------------ timing helpers
+def time_graph(torch, stream, body, launches_per_replay, samples, warm=3, min_launches=32):
+    """Captures `body()` into one CUDA graph; a sample is the graph replayed back to back until it covers at least
+    `min_launches` launches (so that the event records between samples are amortised), bracketed by its own events
+    on `stream`.  Returns the list of microseconds per launch, one entry per sample."""
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g, stream=stream):
+        body()
+    for _ in range(warm):
+        g.replay()
+    stream.synchronize()
+    m = max(1, -(-min_launches // launches_per_replay))
+    evs = [torch.cuda.Event(enable_timing=True) for _ in range(samples + 1)]
+    evs[0].record(stream)
+    for i in range(samples):
+        for _ in range(m):
+            g.replay()
+        evs[i + 1].record(stream)
+    stream.synchronize()
+    return [evs[i].elapsed_time(evs[i + 1]) * 1e3 / (m * launches_per_replay) for i in range(samples)]
+
+
+def stats(us_list):
+    return {"us": statistics.mean(us_list), "us_median": statistics.median(us_list), "us_min": min(us_list),
+            "samples": len(us_list)}
+
+
+def accept_traffic_model(cfg, accept_len):
+    """Bytes of the accept stage from the verdicts of one step (accept_len: int tensor [B] on the host).
+
+    definition : both logit rows of every position, plus the q row of each sequence's first rejection (the rows
+                 the stage's definition needs when every position is examined);
+    chain      : only the positions a sequential chain would look at (up to and including the first rejection),
+                 plus the same q rows — the least any schedule can read.
+    """
+    row = cfg.V_valid * 4
+    rejecting = int((accept_len < cfg.K).sum())
+    examined = int(np.minimum(accept_len + 1, cfg.K).sum())
+    return {"definition": 2 * cfg.B * cfg.K * row + rejecting * row, "chain": 2 * examined * row + rejecting * row,
+            "rejecting_sequences": rejecting, "positions_on_chain": examined}
+
+
+# DRAM bytes of one hawk_cfg_accept call from the ncu captures summarised in profiles/ (rows kernel, read + write)
+ACCEPT_TRAFFIC_BYTES = {}
+
+
+def launches_per_step(cfg, first, sms):
+    """Kernels one verify step launches: attention (+ its merge kernel when items are cut), head (+ a zeroing
+    kernel when its tiles are split along the hidden dimension), accept rows + per-sequence pass (+ a marking
+    kernel from 1.5 waves of rows on)."""
+    head_tiles = -(-cfg.V_valid // 128) * -(-cfg.M // 256)
+    head_split = cfg.M < 512 and 2 * head_tiles <= sms and cfg.hidden // 64 >= 16
+    accept_marks = cfg.B * cfg.K > sms + sms // 2
+    return (2 if first.attn_split else 1) + (2 if head_split else 1) + (3 if accept_marks else 2)
+
+
+def run_config(cid, args, torch, hawk, binding, world, rank, local_rank, dist, headline):
+    """Measures one workload: the step (CUDA-graph replay of the three calls over rotating replicas), each kernel
+    alone, the two-call form, and — for the headline workload — the extras and the end-to-end call."""
     cfg = wl.config(cid)
-    if args.impl == "reference":
-        reference_arm(args, cfg, cid)
-        return
-
-    import torch
-    import paper_2510_25739_b200 as hawk
-    from paper_2510_25739_b200 import binding
-
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    rank = int(os.environ.get("RANK", "0"))
-    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
-    if not torch.cuda.is_available():
-        raise SystemExit("bench.py needs a CUDA device; there is no CPU fallback")
-    torch.cuda.set_device(local_rank)
-    dist = None
-    if world > 1:
-        import torch.distributed as dist
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
-    hawk.load_library()
+    peaks = measured_peaks()
     W = max(args.warmup, 3)
-    K_steps = max(args.steps, 1)
+    K_steps = max(args.steps, 1) if headline else max(20, min(args.steps, 300))
+    sms = torch.cuda.get_device_properties(local_rank).multi_processor_count
 
     # ---- replicas: enough bytes that a step never finds its inputs in L2
     first = Replica(cfg, 1000 * cid + 17 * rank, torch, hawk)
@@ -340,36 +377,20 @@ def main():
     n_rep = min(n_rep, 64)
     reps = [first] + [Replica(cfg, 1000 * cid + 17 * rank + 101 * i, torch, hawk) for i in range(1, n_rep)]
     stream = torch.cuda.Stream()
-    # kernels per step: attention (+ its merge kernel when items are cut), head (+ a zeroing kernel when its tiles
-    # are split along the hidden dimension), accept rows + finalize (+ a marking kernel from 1.5 waves of rows on)
-    sms = torch.cuda.get_device_properties(local_rank).multi_processor_count
-    head_tiles = -(-cfg.V_valid // 128) * -(-cfg.M // 256)
-    head_split = cfg.M < 512 and 2 * head_tiles <= sms and cfg.hidden // 64 >= 16
-    accept_marks = cfg.B * cfg.K > sms + sms // 2
-    launches_per_step = (2 if first.attn_split else 1) + (2 if head_split else 1) + (3 if accept_marks else 2)
+    n_launch = launches_per_step(cfg, first, sms)
 
-    # ---- one CUDA graph per replica: [ev0] attn [ev1] head accept
-    graphs, evs = [], []
-    external_events = bool(args.graph_events)
+    graphs = []
     with torch.cuda.stream(stream):
         for r in reps:                       # warm the kernels (function attributes are set on first use)
             run_attn(cfg, r, hawk); run_head(cfg, r, hawk); run_accept(cfg, r, hawk)
         stream.synchronize()
         for r in reps:
-            e0, ext0 = make_event(torch)
-            e1, ext1 = make_event(torch)
-            external_events &= ext0 and ext1
             g = torch.cuda.CUDAGraph()
             with torch.cuda.graph(g, stream=stream):
-                if external_events:
-                    e0.record()
                 run_attn(cfg, r, hawk)
-                if external_events:
-                    e1.record()
                 run_head(cfg, r, hawk)
                 run_accept(cfg, r, hawk)
             graphs.append(g)
-            evs.append((e0, e1))
 
     def barrier():
         if dist is not None:
@@ -380,20 +401,19 @@ def main():
         uuid = "GPU-" + str(torch.cuda.get_device_properties(local_rank).uuid)
     except Exception:
         uuid = ""
-    sampler = ClockSampler(local_rank, uuid)
+    sampler = ClockSampler(local_rank, uuid) if headline else None
     start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    attn_ms = []
     with torch.cuda.stream(stream):
         for i in range(W):
             graphs[i % n_rep].replay()
         barrier()
-        sampler.start()
+        if sampler:
+            sampler.start()
         start.record(stream)
         for i in range(K_steps):
             graphs[i % n_rep].replay()
         stop.record(stream)
         barrier()
-        sampler.stop()
     elapsed_ms = start.elapsed_time(stop)
     if dist is not None:
         t = torch.tensor([elapsed_ms], device="cuda")
@@ -404,96 +424,26 @@ def main():
     value = positions * world / (ms_per_step * 1e-3)
     status = int(sum(int(r.status.item()) for r in reps))
 
-    # ---- dominant kernel: attention, from the events recorded inside the timed graphs (last round of
-    # replays), else from a loop of attention-only launches on the same stream
-    timing_mode = "events inside the timed step graphs"
-    if external_events:
-        try:
-            attn_ms = [e0.elapsed_time(e1) for (e0, e1) in evs[: min(n_rep, K_steps)]]
-        except Exception:
-            attn_ms = []
-    if not attn_ms:
-        # one CUDA graph holding the attention call of every replica, replayed back to back: the launches of a
-        # call issued one by one from Python cost more host time than the call takes on the device
-        timing_mode = ("CUDA graph of the attention call over the rotating replicas (L2-cold), events around "
-                       "the replays on the bench stream")
-        with torch.cuda.stream(stream):
-            g = torch.cuda.CUDAGraph()
-            with torch.cuda.graph(g, stream=stream):
-                for r in reps:
-                    run_attn(cfg, r, hawk)
-            for _ in range(3):
-                g.replay()
-            stream.synchronize()
-            a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            n = max(3, min(200, K_steps // n_rep + 1))
-            a0.record(stream)
-            for _ in range(n):
-                g.replay()
-            a1.record(stream)
-            stream.synchronize()
-            attn_ms = [a0.elapsed_time(a1) / (n * n_rep)]
-    peaks = measured_peaks()
-    attn_s = statistics.mean(attn_ms) * 1e-3
-    achieved = attn_bytes(cfg) / attn_s / 1e9
-    roofline = {"kernel": "hawk_verify_attn", "bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"],
-                "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"], "peak_source": f"of {peaks['source']}",
-                "traffic": ATTN_TRAFFIC_BYTES.get(cid), "us_per_launch": attn_s * 1e6, "algorithmic_bytes": attn_bytes(cfg),
-                "timing": timing_mode}
-
-    # ---- per-kernel loops (each kernel alone, rotating replicas) for the stage breakdown
-    kernels = {}
+    # ---- each kernel alone: one CUDA graph holding the call for every replica (L2-cold), every replay timed with its
+    # own events on the bench stream (issuing the launches of a call one by one from Python costs more host time
+    # than the call takes on the device); the clock sampler keeps running so that these loops are covered too
+    n_samples = max(5, min(30, K_steps // 4 + 1))
+    kern, warm = {}, {}
     with torch.cuda.stream(stream):
         for name, fn in (("attn", run_attn), ("head", run_head), ("accept", run_accept)):
-            g = torch.cuda.CUDAGraph()
-            with torch.cuda.graph(g, stream=stream):
-                for r in reps:
-                    fn(cfg, r, hawk)
-            for _ in range(3):
-                g.replay()
-            stream.synchronize()
-            a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            n = max(3, min(200, K_steps // n_rep + 1))
-            a0.record(stream)
-            for _ in range(n):
-                g.replay()
-            a1.record(stream)
-            stream.synchronize()
-            kernels[name] = a0.elapsed_time(a1) * 1e3 / (n * n_rep)   # us per launch
-        # the same three with ONE replica repeated: inputs L2-warm where they fit (labelled as such)
-        for name, fn in (("attn", run_attn), ("head", run_head), ("accept", run_accept)):
-            g = torch.cuda.CUDAGraph()
-            with torch.cuda.graph(g, stream=stream):
-                for _ in range(4):
-                    fn(cfg, first, hawk)
-            for _ in range(3):
-                g.replay()
-            stream.synchronize()
-            a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            a0.record(stream)
-            for _ in range(20):
-                g.replay()
-            a1.record(stream)
-            stream.synchronize()
-            kernels[name + "_l2_warm"] = a0.elapsed_time(a1) * 1e3 / 80
-        # the head over ALL columns where only part of the vocabulary is valid (the 65536-entry vocabulary)
-        if cfg.V_valid < cfg.V:
+            kern[name] = stats(time_graph(torch, stream, lambda: [fn(cfg, r, hawk) for r in reps], n_rep, n_samples))
+            # the same call with ONE replica repeated: inputs L2-warm where they fit (labelled as such)
+            warm[name] = statistics.median(time_graph(torch, stream, lambda: [fn(cfg, first, hawk) for _ in range(4)],
+                                                      4, 10))
+        if cfg.V_valid < cfg.V:        # the head over ALL columns where only part of the vocabulary is valid
             full_logits = torch.zeros((cfg.M, cfg.V), dtype=torch.float32, device="cuda")
-            g = torch.cuda.CUDAGraph()
-            with torch.cuda.graph(g, stream=stream):
-                for r in reps:
-                    hawk.head_proj(r.x, r.w, 0, cfg.V, logits=full_logits, dev_status=r.status)
-            for _ in range(3):
-                g.replay()
-            stream.synchronize()
-            a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            a0.record(stream)
-            for _ in range(10):
-                g.replay()
-            a1.record(stream)
-            stream.synchronize()
-            kernels["head_full_vocab"] = a0.elapsed_time(a1) * 1e3 / (10 * n_rep)
+            kern["head_full_vocab"] = stats(time_graph(
+                torch, stream, lambda: [hawk.head_proj(r.x, r.w, 0, cfg.V, logits=full_logits, dev_status=r.status)
+                                        for r in reps], n_rep, 10))
             del full_logits
+    if sampler:
+        sampler.stop()
+
     # ---- the two-call form: guidance combined in the head's epilogue, accept reads one guided row per position
     for r in reps:
         r.guided = torch.zeros((cfg.B, cfg.K, cfg.V), dtype=torch.float32, device="cuda")
@@ -504,21 +454,7 @@ def main():
             run_head_cfg(cfg, r, hawk); run_accept_guided(cfg, r, hawk)
         stream.synchronize()
         for name, fn in (("head_cfg", run_head_cfg), ("accept_guided", run_accept_guided)):
-            g = torch.cuda.CUDAGraph()
-            with torch.cuda.graph(g, stream=stream):
-                for r in reps:
-                    fn(cfg, r, hawk)
-            for _ in range(3):
-                g.replay()
-            stream.synchronize()
-            a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            n = max(3, min(200, K_steps // n_rep + 1))
-            a0.record(stream)
-            for _ in range(n):
-                g.replay()
-            a1.record(stream)
-            stream.synchronize()
-            kernels[name] = a0.elapsed_time(a1) * 1e3 / (n * n_rep)
+            kern[name] = stats(time_graph(torch, stream, lambda: [fn(cfg, r, hawk) for r in reps], n_rep, n_samples))
         graphs2 = []
         for r in reps:
             g = torch.cuda.CUDAGraph()
@@ -539,73 +475,187 @@ def main():
         us_step2 = a0.elapsed_time(a1) * 1e3 / K_steps
     same = all(bool(torch.equal(r.accept_len, r.accept_len2)) and bool(torch.equal(r.out_token, r.out_token2))
                for r in reps)
-    rej = sum(int((r.accept_len < cfg.K).sum().item()) for r in reps) / n_rep
+
+    # ---- bytes, flops, fractions
+    hbm, tens = peaks["hbm_gbs"], peaks["bf16_tflops"]
+    models = [accept_traffic_model(cfg, r.accept_len.cpu().numpy()) for r in reps]
+    acc_def = sum(m["definition"] for m in models) / n_rep
+    acc_chain = sum(m["chain"] for m in models) / n_rep
     mean_len = float(sum(float(r.accept_len.float().mean().item()) for r in reps) / n_rep)
-    q_rows = sum(int(r.accept_len.clamp(max=cfg.K - 1).add(1).sum().item()) for r in reps) / n_rep
+    head_tensor_bound = head_flops(cfg) / (tens * 1e12) > head_bytes(cfg) / (hbm * 1e9)
+
+    def hbm_leg(st, nbytes):
+        return {**st, "bytes": nbytes, "GB/s": nbytes / st["us"] / 1e3, "frac_hbm": nbytes / st["us"] / 1e3 / hbm,
+                "frac_hbm_best": nbytes / st["us_min"] / 1e3 / hbm,
+                "frac_hbm_nominal": nbytes / st["us"] / 1e3 / NOMINAL_HBM_GBS}
+
+    attn = {**hbm_leg(kern["attn"], attn_bytes(cfg)), "bound": "hbm", "frac": None,
+            "us_one_replica_l2_warm": warm["attn"]}
+    attn["frac"] = attn["frac_hbm"]
+    head = {**hbm_leg(kern["head"], head_bytes(cfg)), "flops": head_flops(cfg),
+            "TFLOP/s": head_flops(cfg) / kern["head"]["us"] / 1e6,
+            "frac_tensor": head_flops(cfg) / kern["head"]["us"] / 1e6 / tens,
+            "frac_tensor_sustained_peak": head_flops(cfg) / kern["head"]["us"] / 1e6 / peaks["bf16_tflops_sustained"],
+            "frac_tensor_nominal": head_flops(cfg) / kern["head"]["us"] / 1e6 / NOMINAL_BF16_TFLOPS,
+            "bound": "tensor" if head_tensor_bound else "hbm", "us_one_replica_l2_warm": warm["head"]}
+    head["frac"] = head["frac_tensor"] if head_tensor_bound else head["frac_hbm"]
+    accept = {**hbm_leg(kern["accept"], acc_def), "bound": "hbm", "us_one_replica_l2_warm": warm["accept"],
+              "bytes_counted": "both logit rows of every position + the q row of each sequence's first rejection",
+              "bytes_chain": acc_chain, "frac_hbm_chain_bytes": acc_chain / kern["accept"]["us"] / 1e3 / hbm,
+              "bytes_chain_counted": "only positions up to and including each sequence's first rejection (the least "
+                                     "any schedule reads); rows behind a rejection may or may not be read",
+              "dram_bytes_ncu": ACCEPT_TRAFFIC_BYTES.get(cid),
+              "dram_bytes_ncu_source": "profiles/ (not measured in this run)" if cid in ACCEPT_TRAFFIC_BYTES else None}
+    accept["frac"] = accept["frac_hbm"]
+    floor_us = (attn_bytes(cfg) / hbm + max(head_bytes(cfg) / hbm, head_flops(cfg) / tens / 1e3) + acc_def / hbm) / 1e3
     stage = {
-        "attn": {"us": kernels["attn"], "GB/s": attn_bytes(cfg) / kernels["attn"] / 1e3,
-                 "frac_hbm": attn_bytes(cfg) / kernels["attn"] / 1e3 / peaks["hbm_gbs"],
-                 "frac_hbm_nominal": attn_bytes(cfg) / kernels["attn"] / 1e3 / NOMINAL_HBM_GBS,
-                 "us_one_replica_l2_warm": kernels["attn_l2_warm"]},
-        "head": {"us": kernels["head"], "GB/s": head_bytes(cfg) / kernels["head"] / 1e3,
-                 "frac_hbm": head_bytes(cfg) / kernels["head"] / 1e3 / peaks["hbm_gbs"],
-                 "TFLOP/s": head_flops(cfg) / kernels["head"] / 1e6,
-                 "frac_tensor": head_flops(cfg) / kernels["head"] / 1e6 / peaks["bf16_tflops"],
-                 "frac_hbm_nominal": head_bytes(cfg) / kernels["head"] / 1e3 / NOMINAL_HBM_GBS,
-                 "frac_tensor_nominal": head_flops(cfg) / kernels["head"] / 1e6 / NOMINAL_BF16_TFLOPS,
-                 "us_one_replica_l2_warm": kernels["head_l2_warm"]},
-        "accept": {"us": kernels["accept"], "GB/s": accept_bytes(cfg, cfg.B * cfg.K) / kernels["accept"] / 1e3,
-                   "frac_hbm": accept_bytes(cfg, cfg.B * cfg.K) / kernels["accept"] / 1e3 / peaks["hbm_gbs"],
-                   "frac_hbm_nominal": accept_bytes(cfg, cfg.B * cfg.K) / kernels["accept"] / 1e3 / NOMINAL_HBM_GBS,
-                   "us_one_replica_l2_warm": kernels["accept_l2_warm"],
-                   "bytes_counted": "both logit rows of every position + one q row per position (the definition's rows; in calls of more than 1.5 waves rows behind a known rejection are not read, so fewer bytes move)"},
-        "mean_accept_len": mean_len, "sequences_with_rejection": rej, "q_rows_on_chain": q_rows,
+        "attn": attn, "head": head, "accept": accept, "mean_accept_len": mean_len,
+        "sequences_with_rejection": sum(m["rejecting_sequences"] for m in models) / n_rep,
+        "positions_on_chain": sum(m["positions_on_chain"] for m in models) / n_rep,
+        "step_floor_us": floor_us, "step_frac_of_floor": floor_us / (ms_per_step * 1e3),
         **({"head_full_vocab": {
-            "us": kernels["head_full_vocab"], "columns": cfg.V,
-            "TFLOP/s": 2.0 * cfg.M * cfg.hidden * cfg.V / kernels["head_full_vocab"] / 1e6,
-            "GB/s": (cfg.V * cfg.hidden * 2 + cfg.M * cfg.hidden * 2 + cfg.M * cfg.V * 4) / kernels["head_full_vocab"] / 1e3,
+            **kern["head_full_vocab"], "columns": cfg.V,
+            "TFLOP/s": 2.0 * cfg.M * cfg.hidden * cfg.V / kern["head_full_vocab"]["us"] / 1e6,
             "frac_hbm": (cfg.V * cfg.hidden * 2 + cfg.M * cfg.hidden * 2 + cfg.M * cfg.V * 4)
-                        / kernels["head_full_vocab"] / 1e3 / peaks["hbm_gbs"]}} if "head_full_vocab" in kernels else {}),
+                        / kern["head_full_vocab"]["us"] / 1e3 / hbm}} if "head_full_vocab" in kern else {}),
         "two_call_form": {
             "what": "hawk_head_proj_cfg + hawk_cfg_accept_guided: one guided logits row per position crosses HBM",
-            "head_cfg_us": kernels["head_cfg"], "accept_guided_us": kernels["accept_guided"],
+            "head_cfg": kern["head_cfg"], "accept_guided": kern["accept_guided"],
             "step_us": us_step2, "positions_per_s": positions * world / (us_step2 * 1e-6),
             "same_verdicts_as_three_calls": same},
     }
-
-    # ---- candidate-tree verification (not part of the timed step): a (3, 2, 2) tree, 22 nodes per sequence
-    stage["tree_accept"] = bench_tree(cfg, stream, torch, hawk, peaks, 1000 * cid + 17 * rank)
-    stage["tree_attn"] = bench_tree_attn(cfg, stream, torch, hawk, peaks, 1000 * cid + 17 * rank)
-    stage["pool"] = bench_pool(cfg, stream, torch, hawk, peaks, 1000 * cid + 17 * rank)
+    seed = 1000 * cid + 17 * rank
+    stage["tree_attn"] = bench_tree_attn(cfg, stream, torch, hawk, peaks, seed)
+    stage["tree_accept"] = bench_tree(cfg, stream, torch, hawk, peaks, seed)
+    if headline or cid == 2:
+        stage["pool"] = bench_pool(cfg, stream, torch, hawk, peaks, seed)
     if cid == 2:   # the LlamaGen-XL-shaped workload sweeps the KV length over the image: 120 .. 1144
         stage["attn_kv_sweep"] = {str(L): bench_tree_attn(replace(cfg, L=L), stream, torch, hawk, peaks,
                                                           1000 * cid + L, branching=None)
                                   for L in wl.XL_PREFIX_SWEEP}
-
-    # ---- end to end through hawk_verify_step_host: pinned host inputs, copies inside the timed region
     e2e = None
-    if not args.no_e2e:
-        e2e = bench_e2e(cfg, reps, stream, torch, hawk, binding, world, dist, min(K_steps, 2000), W,
+    if headline and not args.no_e2e:
+        e2e = bench_e2e(cfg, reps, stream, torch, hawk, binding, world, dist, min(K_steps, 500), W,
                         eager=args.e2e_eager)
+    out = {"cid": cid, "cfg": cfg, "value": value, "ms_per_step": ms_per_step, "steps": K_steps, "warmup": W,
+           "positions": positions, "n_rep": n_rep, "replica_bytes": first.bytes(), "launches_per_step": n_launch,
+           "kernels": stage, "status": status, "e2e": e2e, "clocks": sampler.summary() if sampler else None}
+    del graphs, graphs2, reps, first
+    torch.cuda.empty_cache()
+    return out
+
+
+def compact(res):
+    """One workload's entry of `per_config`: the step, the three kernels (mean / median / min microseconds) and each
+    kernel's fraction of the roofline that bounds it."""
+    k = res["kernels"]
+
+    def leg(d, keys):
+        return {key: d[key] for key in keys if key in d}
+
+    kk = ("us", "us_median", "us_min", "bound", "frac", "frac_hbm", "frac_tensor", "bytes", "flops", "frac_hbm_chain_bytes")
+    return {"workload": workload_name(res["cfg"], res["cid"]), "step_us": res["ms_per_step"] * 1e3, "steps": res["steps"],
+            "positions_per_s": res["value"], "attn": leg(k["attn"], kk), "head": leg(k["head"], kk),
+            "accept": leg(k["accept"], kk), "step_floor_us": k["step_floor_us"],
+            "step_frac_of_floor": k["step_frac_of_floor"], "mean_accept_len": k["mean_accept_len"],
+            "two_call_step_us": k["two_call_form"]["step_us"],
+            "same_verdicts_as_three_calls": k["two_call_form"]["same_verdicts_as_three_calls"],
+            "tree_attn": leg(k["tree_attn"], ("us", "frac_hbm")), "tree_accept": leg(k["tree_accept"], ("us", "frac_hbm")),
+            "dev_status": res["status"]}
+
+
+# ------------------------------------------------------------------------------------------ main arm
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=500)
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--config", type=int, default=0,
+                    help="workload id 1..5; default: headline on workload 5 (the largest) plus a per_config table of all five")
+    ap.add_argument("--impl", default="hawk", choices=["hawk", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-per-config", action="store_true")
+    ap.add_argument("--e2e-eager", action="store_true", help="time the end-to-end call eagerly instead of as a graph")
+    args = ap.parse_args()
+    cid = args.config if args.config else HEADLINE_CONFIG
+    cfg = wl.config(cid)
+    if args.impl == "reference":
+        reference_arm(args, cfg, cid)
+        return
+
+    import torch
+    import paper_2510_25739_b200 as hawk
+    from paper_2510_25739_b200 import binding
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device; there is no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    hawk.load_library()
+
+    res = run_config(cid, args, torch, hawk, binding, world, rank, local_rank, dist, headline=True)
+    peaks = measured_peaks()
+    k = res["kernels"]
+    # the dominant kernel of the step: whichever of the three calls takes the largest share of it
+    dom = max(("attn", "head", "accept"), key=lambda n: k[n]["us"])
+    d = k[dom]
+    if d["bound"] == "tensor":
+        roofline = {"kernel": "hawk_head_proj", "bound": "tensor", "achieved": d["TFLOP/s"], "peak": peaks["bf16_tflops"],
+                    "unit": "TFLOP/s", "frac": d["frac_tensor"], "algorithmic_flops": d["flops"], "traffic": None}
+    else:
+        name = {"attn": "hawk_verify_attn", "head": "hawk_head_proj", "accept": "hawk_cfg_accept"}[dom]
+        traffic = ATTN_TRAFFIC_BYTES.get(cid) if dom == "attn" else None
+        roofline = {"kernel": name, "bound": "hbm", "achieved": d["GB/s"], "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                    "frac": d["frac_hbm"], "algorithmic_bytes": d["bytes"], "traffic": traffic,
+                    "traffic_source": ("ncu capture summarised in profiles/ (dram read + write of one call; not "
+                                       "measured in this run)") if traffic else None}
+    roofline.update({"peak_source": f"of {peaks['source']}", "us_per_launch": d["us"], "us_per_launch_median": d["us_median"],
+                     "us_per_launch_min": d["us_min"], "share_of_step": d["us"] / (res["ms_per_step"] * 1e3),
+                     "timing": "CUDA graph of the call over the rotating replicas (L2-cold), every replay bracketed by "
+                               "events on the bench stream"})
+
+    per_config = None
+    if world == 1 and not args.config and not args.no_per_config:
+        per_config = {}
+        for c in (1, 2, 3, 4, 5):
+            per_config[str(c)] = compact(res if c == cid else
+                                         run_config(c, args, torch, hawk, binding, world, rank, local_rank, dist, False))
 
     line = {
-        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K_steps, "warmup": W,
-        "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": "bf16", "data": "synthetic",
-        "config": {"workload": workload_name(cfg, cid), "positions_per_step_per_gpu": positions,
+        "metric": METRIC, "value": res["value"], "unit": UNIT, "n_gpus": world, "steps": res["steps"],
+        "warmup": res["warmup"], "ms_per_step": res["ms_per_step"], "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": workload_name(cfg, cid), "positions_per_step_per_gpu": res["positions"],
                    "arithmetic": "bf16 operands (Q, K, V, X, W), fp32 accumulation, fp32 logits and accept stage",
-                   "l2": f"inputs rotate over {n_rep} replicas ({n_rep * first.bytes() / 1e6:.0f} MB > 3x L2)",
+                   "l2": f"inputs rotate over {res['n_rep']} replicas "
+                         f"({res['n_rep'] * res['replica_bytes'] / 1e6:.0f} MB > 3x L2)",
                    "launch": "one CUDA graph replay per step (3 C-ABI calls captured)",
                    "parallelism": f"{world} independent replicas, sequences sharded, no collective"},
-        "clocks": sampler.summary(), "e2e": e2e, "gpu_launches": launches_per_step * K_steps,
-        "roofline": roofline, "kernels": stage, "dev_status": status,
+        "clocks": res["clocks"], "e2e": res["e2e"], "gpu_launches": res["launches_per_step"] * res["steps"],
+        "roofline": roofline, "kernels": k, "dev_status": res["status"], "per_config": per_config,
     }
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        _, t1, _ = oracle_sample(cfg, wl.seed_for(cid), 1)
-        reps_cpu = max(1, min(2000, int(22.0 / max(t1, 1e-3))))    # 10 to 30 s of CPU work (the first, cold step is the slowest)
-        v, dt, cores = oracle_sample(cfg, wl.seed_for(cid), reps_cpu)
+        seed = wl.seed_for(cid)
+        oracle_sample(replace(cfg, B=min(cfg.B, 2)), seed, 1)        # builds the oracle, warms the page cache
+        _, t1, _ = oracle_sample(cfg, seed, 1)
+        reps_cpu = max(1, min(2000, int(18.0 / max(t1, 1e-3))))      # 10 to 30 s of CPU work in all
+        v, dt, cores = oracle_sample(cfg, seed, reps_cpu)
         line["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle",
                                 "sample": f"{reps_cpu} full steps of the workload ({dt:.1f} s)"}
+        # once single-threaded, on a bounded sample: the first sequences of the workload (the oracle's cost is
+        # linear in the number of sequences)
+        B1 = max(1, min(cfg.B, int(cfg.B * 5.0 / max(t1 * cores, 1e-3))))
+        v1, dt1, c1 = oracle_sample(replace(cfg, B=B1), seed, 1, threads=1)
+        line["cpu_baseline"]["single_thread"] = {
+            "value": v1, "unit": UNIT, "cores": c1,
+            "sample": f"1 step of the first {B1} of {cfg.B} sequences of the workload ({dt1:.1f} s)"}
     if rank == 0:
         print(json.dumps(line))
     if dist is not None:

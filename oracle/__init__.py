@@ -56,10 +56,21 @@ def _c(a, dtype):
     return a
 
 
+def _gomp():
+    return ctypes.CDLL("libgomp.so.1")
+
+
 def threads() -> int:
-    """Threads the OpenMP loops use (OMP_NUM_THREADS if set, else the host's cores)."""
-    env = os.environ.get("OMP_NUM_THREADS")
-    return int(env) if env else (os.cpu_count() or 1)
+    """Threads the OpenMP loops will use (OMP_NUM_THREADS or the host's cores, unless set_threads() changed it)."""
+    _load()
+    return int(_gomp().omp_get_max_threads())
+
+
+def set_threads(n: int) -> None:
+    """Number of threads for the OpenMP loops from now on (timing only: results do not depend on it, every
+    parallel loop runs over independent units)."""
+    _load()
+    _gomp().omp_set_num_threads(int(n))
 
 
 def verify_attn(q, k_cache, v_cache, prefix_len, sm_scale) -> np.ndarray:
