@@ -80,17 +80,9 @@ def test_configs_full_size(config_id):
 
 
 @pytest.mark.parametrize("config_id", [3, 5])
-def test_large_configs_sampled_rows(config_id):
-    """Full-size launch; the oracle checks a sample of token rows (its naive loops are slow)."""
-    import paper_2510_25739_b200 as hawk
+def test_large_configs_full_matrix(config_id):
+    """Full-size launch of the two workloads with the most token rows (384 and 1024: the CTA-pair kernels), every
+    logit compared with the oracle (its naive fp64 loops take a few seconds on the host cores)."""
     cfg = wl.config(config_id)
-    h = wl.make_head_inputs(cfg, wl.seed_for(config_id))
-    logits = hawk.head_proj(bf16_to_torch(h["x"]), bf16_to_torch(h["w"]))
-    torch.cuda.synchronize()
-    rng = np.random.default_rng(config_id)
-    rows = np.unique(np.concatenate([[0, cfg.M - 1, 255, 256], rng.integers(0, cfg.M, 28)]))
-    rows = rows[rows < cfg.M]
-    want = oracle.head_proj(h["x"][rows], h["w"]).astype(np.float64)
-    got = logits[torch.from_numpy(rows).cuda()].cpu().numpy().astype(np.float64)
-    rms = np.sqrt((want ** 2).mean())
-    assert (np.abs(got - want) <= RTOL * np.abs(want) + ATOL_RMS * rms).all()
+    worst = _check(cfg.M, cfg.hidden, cfg.V, cfg.v_begin, cfg.v_end, wl.seed_for(config_id))
+    print(f"config {config_id}: max err / rms = {worst:.2e}")

@@ -46,6 +46,34 @@ def test_matches_the_workspace_call_twice_in_a_row():
         assert int(got_len.min()) >= 0 and int(got_len.max()) <= cfg.K
 
 
+def test_many_rows_twice_with_different_inputs():
+    """A step of 64 sequences x 8 drafts: more than 1.5 rows per SM, so the call first marks every verdict slot of
+    the built-in array unknown and rows behind a rejection return early.  The second step has other inputs and
+    meets the array still holding the first step's verdicts; both must equal the workspace-taking call."""
+    import paper_2510_25739_b200 as hawk
+    import oracle
+    cfg = wl.config(5, top_k=0, q_alpha=0.6)
+    assert cfg.B * cfg.K > 222
+    for seed, bonus in ((4300, False), (4301, True)):
+        args = _step_inputs(cfg, seed, bonus)
+        # drafts that are partly accepted: q mixed with the target distribution (input recipe only; the expected
+        # values below come from the workspace-taking call, not from the oracle)
+        p, _ = oracle.target_probs_rows(args[0].cpu().numpy(), cfg.v_begin, cfg.v_end, cfg.cfg_scale, cfg.temperature,
+                                        cfg.top_k)
+        q = wl.make_q(cfg, seed, np.nan_to_num(p[:, :cfg.K]))
+        args[1], args[2] = to_dev(q), to_dev(wl.draw_drafts(q, seed))
+        params = (cfg.v_begin, cfg.v_end, cfg.cfg_scale, cfg.temperature, cfg.top_k)
+        want_len, want_tok = hawk.cfg_accept(*args, *params, has_bonus_row=bonus)
+        got_len = torch.full((cfg.B,), -7, dtype=torch.int32, device="cuda")
+        got_tok = torch.full((cfg.B,), -7, dtype=torch.int32, device="cuda")
+        status = torch.zeros(1, dtype=torch.int32, device="cuda")
+        hawk.cfg_accept_noalloc(*args, *params, got_len, got_tok, has_bonus_row=bonus, dev_status=status)
+        torch.cuda.synchronize()
+        assert int(status.item()) == 0
+        assert torch.equal(got_len, want_len) and torch.equal(got_tok, want_tok)
+        assert 0 < float(got_len.float().mean()) < cfg.K     # the step has both accepted and rejected drafts
+
+
 def test_step_larger_than_the_builtin_array_is_refused():
     import paper_2510_25739_b200 as hawk
     from paper_2510_25739_b200.binding import HawkError
