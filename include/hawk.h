@@ -15,8 +15,10 @@
  *
  * Conventions common to all entry points
  *   - Every pointer is a DEVICE pointer owned by the caller unless the comment says "host".  The
- *     library allocates nothing, frees nothing, never synchronises and keeps no pointer after
- *     the call returns.  All work is queued on `stream`.
+ *     library allocates no device memory, frees nothing, never synchronises and keeps no pointer
+ *     after the call returns.  All work is queued on `stream`.  (Two calls keep state of their own and
+ *     say so in their comments: hawk_verify_step_host owns one stream and two events per device,
+ *     hawk_cfg_accept_noalloc a fixed array in the library's device image.)
  *   - Tensors are dense, row-major in the index order written in brackets, base address aligned
  *     to 16 bytes.  bf16 is the 16 high bits of an IEEE fp32.
  *   - The return value is the only error channel.  On any error nothing is launched and the
@@ -94,8 +96,8 @@ hawk_status hawk_verify_attn(const void *q, const void *k_cache, const void *v_c
 /* ------------------------------------------------------------------------------------------------
  * hawk_verify_attn_tree - the same attention for a candidate tree.
  *
- * Operation (Sec. 4.2: the candidates of a tree are verified in one forward pass, "akin to tree
- * speculative decoding"): the N tree nodes of a stream are N queries; node i attends to the whole
+ * Operation (Sec. 4.2: all candidates of the tree are verified in one forward pass of the target
+ * model): the N tree nodes of a stream are N queries; node i attends to the whole
  * cached prefix and, inside the block, only to the nodes on its own path from the root:
  *     key j <  prefix_len[s]                  visible to every node
  *     key j == prefix_len[s] + m, 0 <= m < N  visible to node i iff bit m of anc_mask[i] is set
@@ -373,7 +375,15 @@ hawk_status hawk_cfg_accept_noalloc(const float *logits, const float *q_probs, c
  * results are valid after the stream has been synchronised.  Use pinned host memory for the copies
  * to be asynchronous.  The KV cache, the head weight and the prefix lengths are resident device
  * state; all d_* staging and workspaces are device memory owned by the caller.
- * Errors: as the three stage calls, plus HAWK_ERR_CUDA if a copy is refused.
+ * State kept by this call: the first call on a device creates one non-blocking stream and two events
+ * for that device and keeps them until the process exits (no device memory).  Every call on the device
+ * uses them, so the queuing part of a call runs under a per-device mutex: calls from several host
+ * threads are queued one after the other, each correctly ordered against its own `stream`, and the
+ * late copies of steps that are in flight together share the one side stream.
+ * Errors: the argument checks of all three stage calls run before anything is queued, on the staging
+ * pointers and sizes the stages will be given, so a call refused for its arguments (any code but
+ * HAWK_ERR_CUDA) has queued no copy and no kernel.  HAWK_ERR_CUDA means the runtime refused a copy,
+ * an event or a launch after the call had started to queue work.
  * ---------------------------------------------------------------------------------------------- */
 typedef struct {
     /* sizes and sampling parameters */

@@ -25,32 +25,61 @@ def _nvcc() -> str:
     return exe
 
 
-def _stale() -> bool:
-    if not LIB.exists():
-        return True
-    t = LIB.stat().st_mtime
-    deps = list(CSRC.glob("*.cu")) + list(CSRC.glob("*.cuh")) + [PKG.parent / "include" / "hawk.h"]
-    return any(d.stat().st_mtime > t for d in deps)
+def _deps_mtime() -> float:
+    hdrs = list(CSRC.glob("*.cuh")) + [PKG.parent / "include" / "hawk.h"]
+    return max(h.stat().st_mtime for h in hdrs)
 
 
-def build(force: bool = False, verbose: bool = False) -> Path:
-    if not force and not _stale():
-        return LIB
-    tmp = LIB.with_suffix(f".{os.getpid()}.tmp")
-    cmd = [_nvcc(), "-std=c++17", "-O3", "-lineinfo", *ARCH_FLAGS, "-Xcompiler", "-fPIC", "-shared",
-           "-cudart", "static", "-o", str(tmp)]
+def _flags(verbose: bool):
+    flags = ["-std=c++17", "-O3", "-lineinfo", *ARCH_FLAGS, "-Xcompiler", "-fPIC"]
     if verbose:
-        cmd += ["-Xptxas", "-v"]
-    cmd += os.environ.get("HAWK_NVCC_FLAGS", "").split()   # e.g. -DHAWK_ATTN_WARPS=4 -DHAWK_ATTN_STAGE_KB=16
-    cmd += [str(CSRC / s) for s in SOURCES]
-    res = subprocess.run(cmd, capture_output=True, text=True)
+        flags += ["-Xptxas", "-v"]
+    return flags + os.environ.get("HAWK_NVCC_FLAGS", "").split()   # e.g. -DHAWK_ATTN_WARPS=4 -DHAWK_ATTN_STAGE_KB=16
+
+
+def build(force: bool = False, verbose: bool = False, lib: Path = LIB, objdir: Path | None = None) -> Path:
+    """Compiles every source to an object of its own (in parallel; only the ones whose source or headers changed)
+    and links them into `lib`."""
+    objdir = objdir or (PKG / "_build")
+    objdir.mkdir(exist_ok=True)
+    tag = objdir / "flags.txt"
+    flags = _flags(verbose)
+    if not tag.exists() or tag.read_text() != " ".join(flags):
+        force = True
+    hdr_t = _deps_mtime()
+    jobs = []
+    for src in SOURCES:
+        obj = objdir / (Path(src).stem + ".o")
+        s = CSRC / src
+        if force or not obj.exists() or obj.stat().st_mtime < max(s.stat().st_mtime, hdr_t):
+            jobs.append((s, obj))
+    if not jobs and lib.exists() and all(lib.stat().st_mtime >= (objdir / (Path(s).stem + ".o")).stat().st_mtime
+                                         for s in SOURCES):
+        return lib
+    nvcc = _nvcc()
+
+    def compile_one(job):
+        s, obj = job
+        return s, subprocess.run([nvcc, *flags, "-c", str(s), "-o", str(obj)], capture_output=True, text=True)
+
+    from concurrent.futures import ThreadPoolExecutor
+    with ThreadPoolExecutor(max_workers=max(1, min(len(jobs), os.cpu_count() or 1))) as pool:
+        for s, res in pool.map(compile_one, jobs):
+            if res.returncode != 0:
+                sys.stderr.write(res.stdout + res.stderr)
+                raise RuntimeError(f"nvcc failed on {s.name}")
+            if verbose:
+                sys.stderr.write(res.stderr)
+    tag.write_text(" ".join(flags))
+    tmp = lib.with_suffix(f".{os.getpid()}.tmp")
+    objs = [str(objdir / (Path(s).stem + ".o")) for s in SOURCES]
+    res = subprocess.run([nvcc, *ARCH_FLAGS, "-shared", "-cudart", "static", "-o", str(tmp), *objs],
+                         capture_output=True, text=True)
     if res.returncode != 0:
         sys.stderr.write(res.stdout + res.stderr)
-        raise RuntimeError("nvcc failed building libhawk_verify.so")
-    if verbose:
-        sys.stderr.write(res.stderr)
-    os.replace(tmp, LIB)
-    return LIB
+        raise RuntimeError("nvcc failed linking " + lib.name)
+    os.replace(tmp, lib)
+    return lib
 
 
 if __name__ == "__main__":

@@ -945,12 +945,11 @@ extern "C" size_t hawk_cfg_accept_workspace_bytes(int B, int K, int V)
     return static_cast<size_t>(B) * static_cast<size_t>(K + 1) * sizeof(int32_t);
 }
 
-namespace {
-hawk_status cfg_accept_impl(const float *logits, int guided_in, const float *q_probs, const int32_t *draft,
-                            const float *u_accept, const float *u_resample, int B, int K, int V, int v_begin,
-                            int v_end, float cfg_scale, float temperature, int top_k, int has_bonus_row,
-                            int32_t *accept_len, int32_t *out_token, float *p_debug, void *workspace,
-                            size_t workspace_bytes, int32_t *dev_status, hawk_stream_t stream)
+hawk_status hawk_host::check_cfg_accept_args(const float *logits, const float *q_probs, const int32_t *draft,
+                                             const float *u_accept, const float *u_resample, int B, int K, int V,
+                                             int v_begin, int v_end, float cfg_scale, float temperature,
+                                             const int32_t *accept_len, const int32_t *out_token, const float *p_debug,
+                                             const void *workspace, size_t workspace_bytes)
 {
     if (B < 0 || K < 0 || V < 0) return HAWK_ERR_SHAPE;
     if (B == 0) return HAWK_OK;
@@ -967,6 +966,22 @@ hawk_status cfg_accept_impl(const float *logits, int guided_in, const float *q_p
     const size_t need = hawk_cfg_accept_workspace_bytes(B, K, V);
     if (!workspace || workspace_bytes < need) return HAWK_ERR_WORKSPACE;
     if (!hawk_host::aligned16(workspace)) return HAWK_ERR_ALIGN;
+    return HAWK_OK;
+}
+
+namespace {
+hawk_status cfg_accept_impl(const float *logits, int guided_in, const float *q_probs, const int32_t *draft,
+                            const float *u_accept, const float *u_resample, int B, int K, int V, int v_begin,
+                            int v_end, float cfg_scale, float temperature, int top_k, int has_bonus_row,
+                            int32_t *accept_len, int32_t *out_token, float *p_debug, void *workspace,
+                            size_t workspace_bytes, int32_t *dev_status, hawk_stream_t stream)
+{
+    const hawk_status chk = hawk_host::check_cfg_accept_args(logits, q_probs, draft, u_accept, u_resample, B, K, V, v_begin,
+                                                            v_end, cfg_scale, temperature, accept_len, out_token, p_debug,
+                                                            workspace, workspace_bytes);
+    if (chk != HAWK_OK) return chk;
+    if (B == 0) return HAWK_OK;
+    const int n = v_end - v_begin;
     if (!hawk_host::is_sm100(nullptr)) return HAWK_ERR_UNSUPPORTED;
 
     AcceptParams P;

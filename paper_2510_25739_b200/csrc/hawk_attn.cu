@@ -883,13 +883,10 @@ extern "C" size_t hawk_verify_attn_workspace_bytes(int S, int K, int H, int H_kv
     return static_cast<size_t>(pl.workers) * 2 * pl.rows_per_item * (D + 2) * sizeof(float);
 }
 
-namespace {
-
-// Common body of hawk_verify_attn (anc_mask == NULL: causal block) and hawk_verify_attn_tree.
-hawk_status verify_attn_impl(const void *q, const void *k_cache, const void *v_cache, const int32_t *prefix_len,
-                             const uint32_t *anc_mask, void *out, int S, int K, int H, int H_kv, int D, int L_cap,
-                             int max_prefix_len, float sm_scale, void *workspace, size_t workspace_bytes,
-                             int32_t *dev_status, hawk_stream_t stream)
+hawk_status hawk_host::check_verify_attn_args(const void *q, const void *k_cache, const void *v_cache,
+                                              const int32_t *prefix_len, const void *out, int S, int K, int H, int H_kv,
+                                              int D, int L_cap, int max_prefix_len, float sm_scale,
+                                              const void *workspace, size_t workspace_bytes)
 {
     if (S < 0 || K < 0 || H < 0 || H_kv < 0 || D < 0 || L_cap < 0 || max_prefix_len < 0) return HAWK_ERR_SHAPE;
     if (S == 0) return HAWK_OK;
@@ -901,14 +898,28 @@ hawk_status verify_attn_impl(const void *q, const void *k_cache, const void *v_c
     if (!hawk_host::aligned16(q) || !hawk_host::aligned16(k_cache) || !hawk_host::aligned16(v_cache) ||
         !hawk_host::aligned16(out))
         return HAWK_ERR_ALIGN;
-    if (!hawk_host::is_sm100(nullptr)) return HAWK_ERR_UNSUPPORTED;
-
-    const AttnPlan pl = make_plan(S, K, H, H_kv, D, max_prefix_len);
     const size_t need = hawk_verify_attn_workspace_bytes(S, K, H, H_kv, D, max_prefix_len);
     if (need > 0) {
         if (!workspace || workspace_bytes < need) return HAWK_ERR_WORKSPACE;
         if (!hawk_host::aligned16(workspace)) return HAWK_ERR_ALIGN;
     }
+    return HAWK_OK;
+}
+
+namespace {
+
+// Common body of hawk_verify_attn (anc_mask == NULL: causal block) and hawk_verify_attn_tree.
+hawk_status verify_attn_impl(const void *q, const void *k_cache, const void *v_cache, const int32_t *prefix_len,
+                             const uint32_t *anc_mask, void *out, int S, int K, int H, int H_kv, int D, int L_cap,
+                             int max_prefix_len, float sm_scale, void *workspace, size_t workspace_bytes,
+                             int32_t *dev_status, hawk_stream_t stream)
+{
+    const hawk_status chk = hawk_host::check_verify_attn_args(q, k_cache, v_cache, prefix_len, out, S, K, H, H_kv, D, L_cap,
+                                                             max_prefix_len, sm_scale, workspace, workspace_bytes);
+    if (chk != HAWK_OK) return chk;
+    if (S == 0) return HAWK_OK;
+    if (!hawk_host::is_sm100(nullptr)) return HAWK_ERR_UNSUPPORTED;
+    const AttnPlan pl = make_plan(S, K, H, H_kv, D, max_prefix_len);
 
     const int tile_keys = D == 64 ? AttnCfg<64>::kTileKeys : AttnCfg<128>::kTileKeys;
     CUtensorMap map_k, map_v;

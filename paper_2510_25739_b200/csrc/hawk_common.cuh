@@ -431,6 +431,20 @@ bool is_sm100(int *sm_count);
 
 inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
+// The host-side argument checks of the three stage calls, without the device query and without any CUDA call:
+// HAWK_OK means the stage would go on to look at the device and launch.  The stage calls run them first; the
+// host-buffer step call runs all three before it queues its first copy.
+hawk_status check_verify_attn_args(const void *q, const void *k_cache, const void *v_cache, const int32_t *prefix_len,
+                                   const void *out, int S, int K, int H, int H_kv, int D, int L_cap, int max_prefix_len,
+                                   float sm_scale, const void *workspace, size_t workspace_bytes);
+hawk_status check_head_proj_args(const void *x, const void *w, const float *logits, int M, int hidden, int V,
+                                 int v_begin, int v_end);
+hawk_status check_cfg_accept_args(const float *logits, const float *q_probs, const int32_t *draft,
+                                  const float *u_accept, const float *u_resample, int B, int K, int V, int v_begin,
+                                  int v_end, float cfg_scale, float temperature, const int32_t *accept_len,
+                                  const int32_t *out_token, const float *p_debug, const void *workspace,
+                                  size_t workspace_bytes);
+
 // Launches `kernel` with programmatic stream serialisation (see grid_dependency_wait()).
 template <class... KArgs, class... Args>
 inline cudaError_t launch_dependent(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream,

@@ -475,11 +475,8 @@ __global__ void head_zero_kernel(float *logits, int M, int V, int v_begin, int n
 
 }  // namespace
 
-namespace {
-// pairs == 0: logits [M][V]; pairs > 0: M == 2 * pairs and `logits` receives guided rows [pairs][V].
-hawk_status head_proj_impl(const void *x, const void *w, float *logits, int M, int pairs, float cfg_scale,
-                           float temperature, int hidden, int V, int v_begin, int v_end, int32_t *dev_status,
-                           hawk_stream_t stream)
+hawk_status hawk_host::check_head_proj_args(const void *x, const void *w, const float *logits, int M, int hidden, int V,
+                                            int v_begin, int v_end)
 {
     if (M < 0 || hidden < 0 || V < 0) return HAWK_ERR_SHAPE;
     if (v_begin < 0 || v_end > V || v_begin > v_end) return HAWK_ERR_SHAPE;
@@ -487,6 +484,18 @@ hawk_status head_proj_impl(const void *x, const void *w, float *logits, int M, i
     if (!x || !w || !logits) return HAWK_ERR_NULL;
     if (hidden < 64 || hidden % 64 != 0) return HAWK_ERR_UNSUPPORTED;
     if (!hawk_host::aligned16(x) || !hawk_host::aligned16(w) || !hawk_host::aligned16(logits)) return HAWK_ERR_ALIGN;
+    return HAWK_OK;
+}
+
+namespace {
+// pairs == 0: logits [M][V]; pairs > 0: M == 2 * pairs and `logits` receives guided rows [pairs][V].
+hawk_status head_proj_impl(const void *x, const void *w, float *logits, int M, int pairs, float cfg_scale,
+                           float temperature, int hidden, int V, int v_begin, int v_end, int32_t *dev_status,
+                           hawk_stream_t stream)
+{
+    const hawk_status chk = hawk_host::check_head_proj_args(x, w, logits, M, hidden, V, v_begin, v_end);
+    if (chk != HAWK_OK) return chk;
+    if (M == 0 || v_begin == v_end) return HAWK_OK;
     int sm_count = 0;
     if (!hawk_host::is_sm100(&sm_count)) return HAWK_ERR_UNSUPPORTED;
 
@@ -578,8 +587,9 @@ hawk_status head_proj_impl(const void *x, const void *w, float *logits, int M, i
     if (use_pair) {
         // pairs that can be resident at once (an SM without a free neighbour in its group takes none): a
         // persistent grid larger than that would run its last pairs after all the others have finished
-        static int max_pairs_of[64];
-        if (max_pairs_of[device] == 0) {
+        static std::atomic<int> max_pairs_of[64];  // per device, looked up once (two threads may both look it up: same value)
+        int max_pairs = max_pairs_of[device].load(std::memory_order_relaxed);
+        if (max_pairs == 0) {
             cudaLaunchConfig_t occ = {};
             occ.gridDim = dim3(sm_count / 2 * 2);
             occ.blockDim = dim3(kPairThreads);
@@ -589,9 +599,9 @@ hawk_status head_proj_impl(const void *x, const void *w, float *logits, int M, i
                 (void)cudaGetLastError();
                 n = sm_count / 4;  // conservative: half of the SMs
             }
-            max_pairs_of[device] = n < sm_count / 2 ? n : sm_count / 2;
+            max_pairs = n < sm_count / 2 ? n : sm_count / 2;
+            max_pairs_of[device].store(max_pairs, std::memory_order_relaxed);
         }
-        const int max_pairs = max_pairs_of[device];
         const int n_pairs = total_tiles < max_pairs ? total_tiles : max_pairs;
         err = hawk_host::launch_dependent(wide ? head_proj_pair_kernel<true> : head_proj_pair_kernel<false>,
                                           dim3(2 * n_pairs), dim3(kPairThreads), smem_req,

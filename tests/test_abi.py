@@ -136,6 +136,47 @@ def test_step_host_argument_checks(lib):
     assert lib.hawk_verify_step_host(ctypes.byref(a), None) == E_NULL     # no buffers given
 
 
+def test_step_host_checks_every_stage_before_it_queues_anything(lib):
+    """The step call runs the argument checks of all three stages before its first copy: a bad argument of the
+    LAST stage is reported although the first two stages' arguments are fine (the pointers are never touched:
+    every call below is refused on the host)."""
+    def good():
+        a = binding.StepHostArgs()
+        a.B, a.K, a.H, a.H_kv, a.D, a.L_cap, a.max_prefix_len = 2, 4, 16, 16, 64, 132, 128
+        a.V, a.v_begin, a.v_end, a.top_k = 16384, 0, 16384, 1000
+        a.sm_scale, a.cfg_scale, a.temperature = 0.125, 4.0, 1.0
+        for name, _ in binding.StepHostArgs._fields_:
+            if name.startswith(("h_", "d_")) and name != "d_status":
+                setattr(a, name, 0x1000)
+        a.attn_workspace_bytes, a.accept_workspace_bytes = 1 << 20, 1 << 20
+        return a
+
+    def call(**kw):
+        a = good()
+        for k, v in kw.items():
+            setattr(a, k, v)
+        return lib.hawk_verify_step_host(ctypes.byref(a), None)
+
+    # accept stage (the last one)
+    assert call(temperature=0.0) == E_PARAM
+    assert call(cfg_scale=float("nan")) == E_PARAM
+    assert call(K=17, L_cap=200) == E_UNSUP                       # attention takes 17 rows, accept does not
+    assert call(accept_workspace_bytes=4) == E_WS
+    assert call(d_accept_workspace=None) == E_WS
+    assert call(d_q_probs=0x1004) == E_ALIGN
+    assert call(v_begin=10, v_end=10) == E_SHAPE
+    # head projection
+    assert call(H=15) == E_UNSUP                                  # hidden 960 is a multiple of 64, 15 heads of 16 kv heads are not
+    assert call(d_logits=0x1008) == E_ALIGN
+    assert call(v_end=20000) == E_SHAPE
+    # attention
+    assert call(D=96) == E_UNSUP
+    assert call(max_prefix_len=130) == E_SHAPE                    # 130 + 4 rows exceed the cache capacity
+    assert call(sm_scale=0.0) == E_PARAM
+    assert call(H_kv=-1) == E_SHAPE
+    assert call(d_k_cache=0x1002) == E_ALIGN
+
+
 def test_tree_accept_argument_checks(lib):
     p, odd = ctypes.c_void_p(0x1000), ctypes.c_void_p(0x1004)
     f = lib.hawk_tree_accept

@@ -78,6 +78,63 @@ def test_host_step_equals_the_three_calls(config_id, B):
         assert torch.equal(h_len, want_len.cpu()) and torch.equal(h_tok, want_tok.cpu())
 
 
+def test_refused_step_queues_nothing():
+    """A step whose accept-stage argument is bad (temperature 0) is refused before the first copy: the staging
+    buffers, the outputs and the status word keep their sentinels, and the stream has nothing to wait for."""
+    import paper_2510_25739_b200 as hawk
+    from paper_2510_25739_b200 import binding
+    from paper_2510_25739_b200.binding import HawkError
+    cfg = wl.config(1)
+    dev = "cuda"
+    a, h, q, drafts, u = _inputs(cfg, 77)
+    host = dict(q=torch.from_numpy(a["q"].view(np.int16)).pin_memory(), x=torch.from_numpy(h["x"].view(np.int16)).pin_memory(),
+                q_probs=torch.from_numpy(q).pin_memory(), draft=torch.from_numpy(drafts).pin_memory(),
+                u_accept=torch.from_numpy(u["u_accept"]).pin_memory(), u_resample=torch.from_numpy(u["u_resample"]).pin_memory())
+    stage = {k: torch.full_like(v, 21, device=dev) for k, v in host.items()}
+    kc, vc, pl, w = (bf16_to_torch(a["k_cache"]), bf16_to_torch(a["v_cache"]), to_dev(a["prefix_len"]),
+                     bf16_to_torch(h["w"]))
+    attn_out = torch.full((cfg.S, cfg.K, cfg.hidden), 3.0, dtype=torch.bfloat16, device=dev)
+    logits = torch.full((cfg.M, cfg.V), -7.0, dtype=torch.float32, device=dev)
+    d_len = torch.full((cfg.B,), -9, dtype=torch.int32, device=dev)
+    d_tok = torch.full((cfg.B,), -9, dtype=torch.int32, device=dev)
+    h_len = torch.full((cfg.B,), -9, dtype=torch.int32).pin_memory()
+    h_tok = torch.full((cfg.B,), -9, dtype=torch.int32).pin_memory()
+    ws_a = torch.empty(max(16, hawk.verify_attn_workspace_bytes(cfg.S, cfg.K, cfg.H, cfg.H_kv, cfg.D, cfg.L)),
+                       dtype=torch.uint8, device=dev)
+    ws_c = torch.empty(max(16, hawk.cfg_accept_workspace_bytes(cfg.B, cfg.K, cfg.V)), dtype=torch.uint8, device=dev)
+    status = torch.full((1,), 0, dtype=torch.int32, device=dev)
+    s = binding.StepHostArgs()
+    s.B, s.K, s.H, s.H_kv, s.D, s.L_cap, s.max_prefix_len = cfg.B, cfg.K, cfg.H, cfg.H_kv, cfg.D, cfg.L_cap, cfg.L
+    s.V, s.v_begin, s.v_end, s.top_k = cfg.V, cfg.v_begin, cfg.v_end, cfg.top_k
+    s.sm_scale, s.cfg_scale, s.temperature = float(a["sm_scale"]), cfg.cfg_scale, 0.0          # <- refused by the accept stage
+    for name in ("q", "x", "q_probs", "draft", "u_accept", "u_resample"):
+        setattr(s, "h_" + name, host[name].data_ptr())
+        setattr(s, "d_" + name, stage[name].data_ptr())
+    s.h_accept_len, s.h_out_token = h_len.data_ptr(), h_tok.data_ptr()
+    s.d_k_cache, s.d_v_cache, s.d_prefix_len, s.d_w = kc.data_ptr(), vc.data_ptr(), pl.data_ptr(), w.data_ptr()
+    s.d_attn_out, s.d_logits, s.d_accept_len, s.d_out_token = (attn_out.data_ptr(), logits.data_ptr(),
+                                                              d_len.data_ptr(), d_tok.data_ptr())
+    s.d_attn_workspace, s.attn_workspace_bytes = ws_a.data_ptr(), ws_a.numel()
+    s.d_accept_workspace, s.accept_workspace_bytes = ws_c.data_ptr(), ws_c.numel()
+    s.d_status = status.data_ptr()
+    torch.cuda.synchronize()
+    with pytest.raises(HawkError) as err:
+        hawk.verify_step_host(s)
+    assert err.value.code == 6                                   # parameter
+    assert torch.cuda.current_stream().query()                   # nothing was queued behind the synchronize above
+    torch.cuda.synchronize()
+    for k, t in stage.items():
+        assert (t == 21).all(), k                                # no input copy ran
+    assert (attn_out == 3.0).all() and (logits == -7.0).all()
+    assert (d_len == -9).all() and (d_tok == -9).all() and (h_len == -9).all() and (h_tok == -9).all()
+    assert int(status.item()) == 0
+    # and the same arguments with a valid temperature go through
+    s.temperature = cfg.temperature
+    hawk.verify_step_host(s)
+    torch.cuda.synchronize()
+    assert (h_len >= 0).all() and int(status.item()) == 0
+
+
 def test_chained_step_against_chained_oracle():
     """Attention output used as the hidden state (hidden = H * D), its logits verified: GPU chain against
     oracle chain.  Rounding upstream (bf16 attention output) moves logits by parts in a thousand, so a
