@@ -6,6 +6,7 @@ step of the verify path is computed here, and there is no fallback: a missing li
 """
 from __future__ import annotations
 
+import contextlib
 import ctypes
 from pathlib import Path
 from typing import Optional
@@ -69,7 +70,28 @@ def load_library() -> ctypes.CDLL:
         raise RuntimeError(
             f"{_LIB_PATH} is missing: build it with `python -m paper_2510_25739_b200.build` "
             "(or __graft_entry__.build()); there is no fallback path")
-    lib = ctypes.CDLL(str(_LIB_PATH))
+    _lib = _open(_LIB_PATH)
+    return _lib
+
+
+@contextlib.contextmanager
+def alternate_library(path):
+    """Routes every call of this module to another build of the same library while the block runs (the tests of
+    the kernels' give-up paths load a variant with short waits this way); the regular library is back afterwards."""
+    global _lib
+    if not Path(path).exists():
+        raise RuntimeError(f"{path} is missing")
+    saved = _lib
+    _lib = _open(Path(path))
+    try:
+        yield _lib
+    finally:
+        _lib = saved
+
+
+def _open(path: Path) -> ctypes.CDLL:
+    """dlopens one build of the library and declares the argument types of its entry points."""
+    lib = ctypes.CDLL(str(path))
     vp, i32, f32, sz = ctypes.c_void_p, ctypes.c_int, ctypes.c_float, ctypes.c_size_t
     lib.hawk_status_string.restype = ctypes.c_char_p
     lib.hawk_status_string.argtypes = [i32]
@@ -119,7 +141,6 @@ def load_library() -> ctypes.CDLL:
     lib.hawk_pool_sample.argtypes = [vp] * 4 + [i32] * 6 + [vp, sz, vp, vp]
     lib.hawk_verify_step_host.restype = i32
     lib.hawk_verify_step_host.argtypes = [ctypes.POINTER(StepHostArgs), vp]
-    _lib = lib
     return lib
 
 

@@ -30,20 +30,22 @@ def _deps_mtime() -> float:
     return max(h.stat().st_mtime for h in hdrs)
 
 
-def _flags(verbose: bool):
+def _flags(verbose: bool, extra=()):
     flags = ["-std=c++17", "-O3", "-lineinfo", *ARCH_FLAGS, "-Xcompiler", "-fPIC"]
     if verbose:
         flags += ["-Xptxas", "-v"]
+    flags += list(extra)
     return flags + os.environ.get("HAWK_NVCC_FLAGS", "").split()   # e.g. -DHAWK_ATTN_WARPS=4 -DHAWK_ATTN_STAGE_KB=16
 
 
-def build(force: bool = False, verbose: bool = False, lib: Path = LIB, objdir: Path | None = None) -> Path:
+def build(force: bool = False, verbose: bool = False, lib: Path = LIB, objdir: Path | None = None,
+          extra_flags=()) -> Path:
     """Compiles every source to an object of its own (in parallel; only the ones whose source or headers changed)
     and links them into `lib`."""
     objdir = objdir or (PKG / "_build")
     objdir.mkdir(exist_ok=True)
     tag = objdir / "flags.txt"
-    flags = _flags(verbose)
+    flags = _flags(verbose, extra_flags)
     if not tag.exists() or tag.read_text() != " ".join(flags):
         force = True
     hdr_t = _deps_mtime()
@@ -80,6 +82,16 @@ def build(force: bool = False, verbose: bool = False, lib: Path = LIB, objdir: P
         raise RuntimeError("nvcc failed linking " + lib.name)
     os.replace(tmp, lib)
     return lib
+
+
+STALL_LIB = PKG / "libhawk_verify_stall.so"
+
+
+def build_stall_variant(force: bool = False) -> Path:
+    """The library the give-up tests load: every wait limited to 2 ms, and one stage per kernel armed for more
+    bytes than its copies deliver (HAWK_TEST_STALL), so that exactly one wait per launch runs out."""
+    return build(force=force, lib=STALL_LIB, objdir=PKG / "_build_stall",
+                 extra_flags=("-DHAWK_WAIT_NS=2000000ull", "-DHAWK_TEST_STALL"))
 
 
 if __name__ == "__main__":

@@ -1035,6 +1035,7 @@ extern "C" hawk_status hawk_cfg_accept(const float *logits, const float *q_probs
                                        void *workspace, size_t workspace_bytes, int32_t *dev_status,
                                        hawk_stream_t stream)
 {
+    const hawk_host::NvtxRange nvtx_range("hawk_cfg_accept");
     return cfg_accept_impl(logits, 0, q_probs, draft, u_accept, u_resample, B, K, V, v_begin, v_end, cfg_scale,
                            temperature, top_k, has_bonus_row, accept_len, out_token, p_debug, workspace,
                            workspace_bytes, dev_status, stream);
@@ -1047,6 +1048,7 @@ extern "C" hawk_status hawk_cfg_accept_guided(const float *guided, const float *
                                               void *workspace, size_t workspace_bytes, int32_t *dev_status,
                                               hawk_stream_t stream)
 {
+    const hawk_host::NvtxRange nvtx_range("hawk_cfg_accept_guided");
     return cfg_accept_impl(guided, 1, q_probs, draft, u_accept, u_resample, B, K, V, v_begin, v_end, 1.0f, 1.0f, top_k,
                            has_bonus_row, accept_len, out_token, p_debug, workspace, workspace_bytes, dev_status,
                            stream);
@@ -1140,6 +1142,7 @@ extern "C" hawk_status hawk_tree_accept(const float *logits, const float *q_prob
                                         int32_t *accept_len, int32_t *out_token, int32_t *path, void *workspace,
                                         size_t workspace_bytes, int32_t *dev_status, hawk_stream_t stream)
 {
+    const hawk_host::NvtxRange nvtx_range("hawk_tree_accept");
     return tree_accept_impl(logits, 0, q_probs, node_token, node_q, child_begin, u_accept, u_resample, B, N, NQ, V,
                             v_begin, v_end, cfg_scale, temperature, top_k, max_depth, accept_len, out_token, path,
                             workspace, workspace_bytes, dev_status, stream);
@@ -1153,6 +1156,7 @@ extern "C" hawk_status hawk_tree_accept_guided(const float *guided, const float 
                                                void *workspace, size_t workspace_bytes, int32_t *dev_status,
                                                hawk_stream_t stream)
 {
+    const hawk_host::NvtxRange nvtx_range("hawk_tree_accept_guided");
     return tree_accept_impl(guided, 1, q_probs, node_token, node_q, child_begin, u_accept, u_resample, B, N, NQ, V,
                             v_begin, v_end, 1.0f, 1.0f, top_k, max_depth, accept_len, out_token, path, workspace,
                             workspace_bytes, dev_status, stream);
@@ -1170,6 +1174,7 @@ extern "C" hawk_status hawk_pool_sample(const float *pool_q, const float *u, con
                                         void *workspace, size_t workspace_bytes, int32_t *dev_status,
                                         hawk_stream_t stream)
 {
+    const hawk_host::NvtxRange nvtx_range("hawk_pool_sample");
     if (B < 0 || NQ < 0 || N < 0 || V < 0) return HAWK_ERR_SHAPE;
     if (B == 0) return HAWK_OK;
     if (!pool_q || !u || !node_q || !node_token) return HAWK_ERR_NULL;
@@ -1239,6 +1244,7 @@ extern "C" hawk_status hawk_cfg_accept_noalloc(const float *logits, const float 
                                                int top_k, int has_bonus_row, int32_t *accept_len,
                                                int32_t *out_token, int32_t *dev_status, hawk_stream_t stream)
 {
+    const hawk_host::NvtxRange nvtx_range("hawk_cfg_accept_noalloc");
     if (B < 0 || K < 0 || V < 0) return HAWK_ERR_SHAPE;
     if (B == 0) return HAWK_OK;
     if (K < 1 || K > 16) return HAWK_ERR_UNSUPPORTED;

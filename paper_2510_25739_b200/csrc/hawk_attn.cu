@@ -214,7 +214,9 @@ __global__ void __launch_bounds__(kWarps * 32, kWarps == kWarpsGroup ? 3 : 1) at
         if (lane == 0) {
             uint8_t *kd = ring + st * kStageBytes;
             uint8_t *vd = kd + C::kHalves * C::kSubTileBytes;
-            mbar_arrive_expect_tx(&full_bar[st], kStageBytes);
+            // (test builds only: the first tile of the first share is armed for more bytes than arrive)
+            const bool stall = kTestStallBytes != 0 && blockIdx.x == 0 && warp == 0 && c.f == f_begin;
+            mbar_arrive_expect_tx(&full_bar[st], kStageBytes + (stall ? kTestStallBytes : 0u));
             const int y = c.row_base + c.tile * TK;
 #pragma unroll
             for (int hf = 0; hf < C::kHalves; ++hf) {
@@ -1002,6 +1004,7 @@ extern "C" hawk_status hawk_verify_attn(const void *q, const void *k_cache, cons
                                         int L_cap, int max_prefix_len, float sm_scale, void *workspace,
                                         size_t workspace_bytes, int32_t *dev_status, hawk_stream_t stream)
 {
+    const hawk_host::NvtxRange nvtx_range("hawk_verify_attn");
     return verify_attn_impl(q, k_cache, v_cache, prefix_len, nullptr, out, S, K, H, H_kv, D, L_cap, max_prefix_len,
                             sm_scale, workspace, workspace_bytes, dev_status, stream);
 }
@@ -1012,6 +1015,7 @@ extern "C" hawk_status hawk_verify_attn_tree(const void *q, const void *k_cache,
                                              float sm_scale, void *workspace, size_t workspace_bytes,
                                              int32_t *dev_status, hawk_stream_t stream)
 {
+    const hawk_host::NvtxRange nvtx_range("hawk_verify_attn_tree");
     if (S > 0 && !anc_mask) return HAWK_ERR_NULL;
     return verify_attn_impl(q, k_cache, v_cache, prefix_len, anc_mask, out, S, N, H, H_kv, D, L_cap, max_prefix_len,
                             sm_scale, workspace, workspace_bytes, dev_status, stream);

@@ -14,7 +14,19 @@
 
 namespace hawk {
 
-constexpr unsigned long long kWaitNs = 1000ull * 1000ull * 1000ull;  // 1 s per wait, at most
+// Time limit of every wait, in nanoseconds.  The tests of the give-up paths build a second library with a
+// limit of a few milliseconds and with HAWK_TEST_STALL (one stage per kernel is armed for 16 bytes more than
+// its copies deliver, so that its wait runs out: nothing faults, nothing hangs, the kernel reports
+// HAWK_DEV_TIMEOUT and leaves through the same path a real stall would take).
+#ifndef HAWK_WAIT_NS
+#define HAWK_WAIT_NS 1000000000ull
+#endif
+constexpr unsigned long long kWaitNs = HAWK_WAIT_NS;  // 1 s per wait unless built otherwise
+#ifdef HAWK_TEST_STALL
+constexpr uint32_t kTestStallBytes = 16;
+#else
+constexpr uint32_t kTestStallBytes = 0;
+#endif
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p)
 {
@@ -419,7 +431,25 @@ __device__ __forceinline__ float warp_sum(float v)
 }  // namespace hawk
 
 // ---------------------------------------------------------------------------------- host side
+#ifndef HAWK_NO_NVTX
+#include <nvtx3/nvToolsExt.h>
+#endif
+
 namespace hawk_host {
+
+// A named range on the calling host thread for the time an entry point spends queuing its work; profilers that
+// follow NVTX attribute the kernels launched inside it to the call.  Without a profiler attached it costs one
+// indirect call.  (NVTX 3 is header-only; nothing is linked.)
+struct NvtxRange {
+#ifndef HAWK_NO_NVTX
+    explicit NvtxRange(const char *name) { nvtxRangePushA(name); }
+    ~NvtxRange() { nvtxRangePop(); }
+#else
+    explicit NvtxRange(const char *) {}
+#endif
+    NvtxRange(const NvtxRange &) = delete;
+    NvtxRange &operator=(const NvtxRange &) = delete;
+};
 
 // Encodes a 2-D bf16 tensor map [rows][cols] (cols contiguous) with a box of box_rows x 64 columns
 // and the 128-byte swizzle.  Uses cuTensorMapEncodeTiled through the runtime's driver entry point,

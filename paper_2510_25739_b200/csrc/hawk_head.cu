@@ -177,7 +177,9 @@ __global__ void __launch_bounds__(kHeadThreads, 1) head_proj_kernel(const __grid
                     ok = mbar_wait(&empty_bar[st], ph ^ 1u, abort_flag);
                     if (!ok) break;
                     uint8_t *a = smem + static_cast<size_t>(st) * P.stage_bytes;
-                    mbar_arrive_expect_tx(&full_bar[st], tx_bytes);
+                    // (test builds only: the first stage of block 0 is armed for more bytes than arrive)
+                    const bool stall = kTestStallBytes != 0 && blockIdx.x == 0 && issued == 0;
+                    mbar_arrive_expect_tx(&full_bar[st], tx_bytes + (stall ? kTestStallBytes : 0u));
                     tma_load_2d(a, &map_w, kb * kBK, row_w, &full_bar[st]);
                     if (P.pairs == 0) {
                         tma_load_2d(a + kATileBytes, &map_x, kb * kBK, row_x, &full_bar[st]);
@@ -361,7 +363,9 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kPairThreads, 1)
                     ok = mbar_wait_cluster(&empty_bar[st], ph ^ 1u, abort_flag);
                     if (!ok) break;
                     uint8_t *a = smem + static_cast<size_t>(st) * P.stage_bytes;
-                    if (rank == 0) mbar_arrive_expect_tx(&full_bar[st], 2 * tx_bytes);  // both CTAs' halves
+                    // (test builds only: the first stage of pair 0 is armed for more bytes than arrive)
+                    const bool stall = kTestStallBytes != 0 && pair == 0 && tile == pair && kb == 0;
+                    if (rank == 0) mbar_arrive_expect_tx(&full_bar[st], 2 * tx_bytes + (stall ? kTestStallBytes : 0u));  // both CTAs' halves
                     const uint32_t bar0 = map_shared_to_cta(&full_bar[st], 0);
                     tma_load_2d_pair(a, &map_w, kb * kBK, row_w, bar0);
                     tma_load_2d_pair(a + kATileBytes, &map_x, kb * kBK, row_x, bar0);
@@ -619,6 +623,7 @@ hawk_status head_proj_impl(const void *x, const void *w, float *logits, int M, i
 extern "C" hawk_status hawk_head_proj(const void *x, const void *w, float *logits, int M, int hidden, int V,
                                       int v_begin, int v_end, int32_t *dev_status, hawk_stream_t stream)
 {
+    const hawk_host::NvtxRange nvtx_range("hawk_head_proj");
     return head_proj_impl(x, w, logits, M, 0, 1.0f, 1.0f, hidden, V, v_begin, v_end, dev_status, stream);
 }
 
@@ -626,6 +631,7 @@ extern "C" hawk_status hawk_head_proj_cfg(const void *x, const void *w, float *g
                                           int V, int v_begin, int v_end, float cfg_scale, float temperature,
                                           int32_t *dev_status, hawk_stream_t stream)
 {
+    const hawk_host::NvtxRange nvtx_range("hawk_head_proj_cfg");
     if (B < 0 || rows < 0) return HAWK_ERR_SHAPE;
     if (static_cast<long long>(B) * rows > (1 << 29)) return HAWK_ERR_UNSUPPORTED;
     if (!(temperature == temperature) || !(cfg_scale == cfg_scale) || isinf(temperature) || isinf(cfg_scale) ||

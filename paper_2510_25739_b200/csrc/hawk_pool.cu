@@ -96,6 +96,7 @@ extern "C" int hawk_spec_cache_slot(int IW, int VSD, int position, int depth)
 
 extern "C" hawk_status hawk_spec_cache_clear(int32_t *cache_tags, int B, int IW, int VSD, hawk_stream_t stream)
 {
+    const hawk_host::NvtxRange nvtx_range("hawk_spec_cache_clear");
     if (B < 0 || IW < 1 || VSD < 1) return HAWK_ERR_SHAPE;
     if (B == 0) return HAWK_OK;
     if (!cache_tags) return HAWK_ERR_NULL;
@@ -108,6 +109,7 @@ extern "C" hawk_status hawk_spec_cache_clear(int32_t *cache_tags, int B, int IW,
 extern "C" hawk_status hawk_spec_cache_put(const float *q_vert, const int32_t *position, float *cache_rows,
                                            int32_t *cache_tags, int B, int IW, int VSD, int V, hawk_stream_t stream)
 {
+    const hawk_host::NvtxRange nvtx_range("hawk_spec_cache_put");
     if (B < 0 || IW < 1 || VSD < 1 || V < 1) return HAWK_ERR_SHAPE;
     if (B == 0) return HAWK_OK;
     if (!q_vert || !position || !cache_rows || !cache_tags) return HAWK_ERR_NULL;
@@ -126,6 +128,7 @@ extern "C" hawk_status hawk_pool_build(const float *q_horiz, const float *cache_
                                        const int32_t *position, float *pool_q, int32_t *pool_source, int B, int K,
                                        int IW, int VSD, int V, hawk_stream_t stream)
 {
+    const hawk_host::NvtxRange nvtx_range("hawk_pool_build");
     if (B < 0 || K < 0 || IW < 1 || VSD < 1 || V < 1) return HAWK_ERR_SHAPE;
     if (B == 0 || K == 0) return HAWK_OK;
     if (!q_horiz || !cache_rows || !cache_tags || !position || !pool_q) return HAWK_ERR_NULL;

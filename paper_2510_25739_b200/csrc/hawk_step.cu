@@ -58,6 +58,7 @@ SideLane *side_lane()
 
 extern "C" hawk_status hawk_verify_step_host(const hawk_step_host_args *a, hawk_stream_t stream)
 {
+    const hawk_host::NvtxRange nvtx_range("hawk_verify_step_host");
     if (!a) return HAWK_ERR_NULL;
     if (a->B < 0 || a->K < 0 || a->H < 0 || a->H_kv < 0 || a->D < 0 || a->V < 0 || a->L_cap < 0 ||
         a->max_prefix_len < 0)
