@@ -86,13 +86,13 @@ def verify_attn(q, k_cache, v_cache, prefix_len, sm_scale) -> np.ndarray:
 
 
 def verify_attn_tree(q, k_cache, v_cache, prefix_len, anc_mask, sm_scale) -> np.ndarray:
-    """q [S,N,H,D], caches [S,H_kv,L_cap,D] (uint16 bf16 bits), prefix_len [S], anc_mask uint32 [N]
+    """q [S,N,H,D], caches [S,H_kv,L_cap,D] (uint16 bf16 bits), prefix_len [S], anc_mask uint64 [N] (N <= 64)
     -> fp64 [S,N,H*D]; node i sees the prefix and the block rows whose bit is set in anc_mask[i]."""
     q = _c(q, np.uint16); k_cache = _c(k_cache, np.uint16); v_cache = _c(v_cache, np.uint16)
-    prefix_len = _c(prefix_len, np.int32); anc_mask = _c(anc_mask, np.uint32)
+    prefix_len = _c(prefix_len, np.int32); anc_mask = _c(anc_mask, np.uint64)
     S, N, H, D = q.shape
     _, H_kv, L_cap, _ = k_cache.shape
-    assert anc_mask.shape == (N,) and N <= 32
+    assert anc_mask.shape == (N,) and N <= 64
     out = np.empty((S, N, H * D), dtype=np.float64)
     _load().hawk_oracle_verify_attn_tree(_p(q), _p(k_cache), _p(v_cache), _p(prefix_len), _p(anc_mask), _p(out),
                                          S, N, H, H_kv, D, L_cap, ctypes.c_double(float(sm_scale)))

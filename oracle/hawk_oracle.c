@@ -426,19 +426,19 @@ int hawk_oracle_tree_accept(const float *logits, const float *q_probs, const int
 }
 
 /* ------------------------------------------------------------------------------------------
- * Step 1 for a candidate tree (Sec. 4.2: "a tree structure is employed to expand the number of
- * candidates that can be verified simultaneously"; verification is "akin to tree speculative
- * decoding"): the N tree nodes of a stream are N queries in one forward pass; node i attends to the
- * whole cached prefix and, inside the block, only to the nodes on its own path from the root.
+ * Step 1 for a candidate tree (Sec. 4.2: the candidates form a tree so that more of them can be
+ * verified at once, all in one forward pass of the target model): the N tree nodes of a stream are N
+ * queries; node i attends to the whole cached prefix and, inside the block, only to the nodes on its
+ * own path from the root.
  * Plain definition of masked softmax attention:
  *   key j <  prefix_len[s]                      visible to every node
  *   key j =  prefix_len[s] + m, 0 <= m < N      visible to node i iff bit m of anc_mask[i] is set
  * (node i's own key/value row is cache row prefix_len[s] + i; anc_mask[i] has bit i set).
  * The chain of K drafts is the tree with anc_mask[i] = 2^(i+1) - 1.
- *   q bf16 [S][N][H][D]; caches bf16 [S][H_kv][L_cap][D]; anc_mask uint32 [N]; out fp64 [S][N][H*D]
+ *   q bf16 [S][N][H][D]; caches bf16 [S][H_kv][L_cap][D]; anc_mask uint64 [N], N <= 64; out fp64 [S][N][H*D]
  * ------------------------------------------------------------------------------------------ */
 void hawk_oracle_verify_attn_tree(const uint16_t *q, const uint16_t *k_cache, const uint16_t *v_cache,
-                                  const int32_t *prefix_len, const uint32_t *anc_mask, double *out,
+                                  const int32_t *prefix_len, const uint64_t *anc_mask, double *out,
                                   int S, int N, int H, int H_kv, int D, int L_cap, double sm_scale)
 {
     int group = H / H_kv;
@@ -454,7 +454,7 @@ void hawk_oracle_verify_attn_tree(const uint16_t *q, const uint16_t *k_cache, co
                 const uint16_t *qv = q + (((size_t)s * N + i) * H + h) * (size_t)D;
                 double m = -INFINITY;
                 for (int j = 0; j < n; ++j) {
-                    int visible = j < pl || ((anc_mask[i] >> (j - pl)) & 1u);
+                    int visible = j < pl || (int)((anc_mask[i] >> (j - pl)) & 1u);
                     if (!visible) {
                         e[j] = -INFINITY;
                         continue;

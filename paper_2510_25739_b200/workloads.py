@@ -254,20 +254,27 @@ def make_tree(branching=(3, 2, 2)) -> dict:
 
 
 def tree_ancestor_masks(child_begin: np.ndarray) -> np.ndarray:
-    """anc_mask[i] (uint32): bit m set iff node m lies on the path from the root to node i, i included.
-    Index bookkeeping for the attention mask of a tree with at most 32 nodes."""
+    """anc_mask[i] (uint64): bit m set iff node m lies on the path from the root to node i, i included.
+    Index bookkeeping for the attention mask of a tree with at most 64 nodes."""
     N = len(child_begin) - 1
+    if N > 64:
+        raise ValueError("a mask word holds 64 nodes")
     parent = np.full(N, -1, np.int64)
     for n in range(N):
         parent[child_begin[n]:child_begin[n + 1]] = n
-    masks = np.zeros(N, np.uint32)
+    masks = np.zeros(N, np.uint64)
     for i in range(N):
         m, n = 0, i
         while n >= 0:
-            m |= 1 << n
+            m |= 1 << int(n)
             n = parent[n]
-        masks[i] = m
+        masks[i] = np.uint64(m)
     return masks
+
+
+def chain_masks(K: int) -> np.ndarray:
+    """The masks of a plain chain of K drafts: position i sees block rows 0..i."""
+    return np.array([(1 << (i + 1)) - 1 for i in range(K)], dtype=np.uint64)
 
 
 def draw_tree_tokens(q: np.ndarray, tree: dict, seed: int) -> np.ndarray:

@@ -35,6 +35,10 @@ def _brute_force(q, kc, vc, prefix, masks, scale):
     ((3, 2), 1, 4, 2, 16, [6]),
     ((2, 2, 2), 2, 1, 1, 8, [9, 4]),
     ((3, 2, 2), 1, 2, 1, 8, [5]),
+    ((3, 3, 3), 1, 2, 2, 8, [7]),          # 40 nodes: masks past the 32nd bit
+    ((4, 3, 2), 2, 2, 1, 8, [3, 11]),      # 41 nodes
+    ((2, 2, 2, 2, 2), 1, 1, 1, 8, [2]),    # 63 nodes
+    ((7, 8), 1, 2, 2, 8, [0]),             # 64 nodes, no prefix at all
 ])
 def test_matches_brute_force(branching, S, H, H_kv, D, prefix):
     tree = wl.make_tree(branching)
@@ -52,13 +56,38 @@ def test_ancestor_masks_of_a_known_tree():
     assert masks.tolist() == [0b1, 0b11, 0b101, 0b1011, 0b10011, 0b100101, 0b1000101]
 
 
-def test_chain_mask_reproduces_causal_attention():
-    rng = np.random.default_rng(5)
-    K = 5
-    q, kc, vc, pl = _rand_case(rng, 2, K, 3, 3, 16, 20, [12, 7])
-    masks = np.array([(2 << i) - 1 for i in range(K)], np.uint32)
+@pytest.mark.parametrize("K", [5, 33, 40, 64])
+def test_chain_mask_reproduces_causal_attention(K):
+    rng = np.random.default_rng(5 + K)
+    q, kc, vc, pl = _rand_case(rng, 2, K, 3, 3, 16, 15 + K, [12, 7])
+    masks = wl.chain_masks(K)
+    assert masks.dtype == np.uint64 and int(masks[-1]) == (1 << K) - 1
     np.testing.assert_array_equal(oracle.verify_attn_tree(q, kc, vc, pl, masks, 0.25),
                                   oracle.verify_attn(q, kc, vc, pl, 0.25))
+
+
+def test_high_mask_bits_matter():
+    """A 40-node tree: clearing bit 35 of node 39's mask (an ancestor past the 32nd row) changes node 39 and nothing
+    else; a mask type narrower than 64 bits would drop that bit silently."""
+    tree = wl.make_tree((3, 3, 3))
+    masks = wl.tree_ancestor_masks(tree["child_begin"])
+    N = tree["N"]
+    assert N == 40
+    node = 39
+    anc = [m for m in range(N) if (int(masks[node]) >> m) & 1]
+    assert max(a for a in anc if a != node) >= 12        # its parent is a depth-2 node
+    # give node 39 one more visible row past bit 32 instead: row 35 (not an ancestor)
+    assert not (int(masks[node]) >> 35) & 1
+    rng = np.random.default_rng(11)
+    q, kc, vc, pl = _rand_case(rng, 1, N, 1, 1, 8, 3 + N, [3])
+    base = oracle.verify_attn_tree(q, kc, vc, pl, masks, 0.4)
+    m2 = masks.copy()
+    m2[node] = np.uint64(int(m2[node]) | (1 << 35))
+    other = oracle.verify_attn_tree(q, kc, vc, pl, m2, 0.4)
+    assert not np.array_equal(base[:, node], other[:, node])
+    keep = [i for i in range(N) if i != node]
+    np.testing.assert_array_equal(base[:, keep], other[:, keep])
+    np.testing.assert_allclose(other, _brute_force(q, kc, vc, pl, m2, 0.4), rtol=1e-12, atol=1e-13)
 
 
 def test_rows_off_the_path_do_not_reach_a_node():
