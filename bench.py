@@ -789,7 +789,7 @@ def bench_tree_attn(cfg, stream, torch, hawk, peaks, seed, branching=(3, 2, 2)):
     else:
         tree = wl.make_tree(branching)
         N = tree["N"]
-        masks = torch.from_numpy(wl.tree_ancestor_masks(tree["child_begin"]).view(np.int32)).cuda()
+        masks = torch.from_numpy(wl.tree_ancestor_masks(tree["child_begin"]).view(np.int64)).cuda()
     dev = torch.device("cuda")
     gen = torch.Generator(device=dev)
     gen.manual_seed(seed + 9)

@@ -82,7 +82,7 @@ int hawk_version(void); /* major*10000 + minor*100 + patch */
  *   workspace    scratch of at least hawk_verify_attn_workspace_bytes(...) bytes, 16-byte aligned;
  *                may be NULL when that function returns 0.  Contents need no initialisation and
  *                are garbage afterwards.
- * Supported: D in {64, 128}; 1 <= K <= 32; H a multiple of H_kv; S*H_kv*L_cap < 2^31.
+ * Supported: D in {64, 128}; 1 <= K <= 64; H a multiple of H_kv; S*H_kv*L_cap < 2^31.
  * Errors: NULL, SHAPE (negative sizes, max_prefix_len + K > L_cap), ALIGN, UNSUPPORTED, WORKSPACE,
  * PARAM (sm_scale not a positive finite number), CUDA.  S == 0 returns HAWK_OK without a launch.
  * ---------------------------------------------------------------------------------------------- */
@@ -105,13 +105,13 @@ hawk_status hawk_verify_attn(const void *q, const void *k_cache, const void *v_c
  * hawk_verify_attn is the special case anc_mask[i] = 2^(i+1) - 1.
  *
  *   q         bf16 [S][N][H][D]
- *   anc_mask  uint32 [N], device memory, shared by all streams
+ *   anc_mask  uint64 [N], device memory, shared by all streams
  *   out       bf16 [S][N][H*D]
  * Everything else, the workspace (hawk_verify_attn_workspace_bytes with K = N) and the errors are
- * those of hawk_verify_attn; 1 <= N <= 32.
+ * those of hawk_verify_attn; 1 <= N <= 64.
  * ---------------------------------------------------------------------------------------------- */
 hawk_status hawk_verify_attn_tree(const void *q, const void *k_cache, const void *v_cache,
-                                  const int32_t *prefix_len, const uint32_t *anc_mask, void *out, int S,
+                                  const int32_t *prefix_len, const uint64_t *anc_mask, void *out, int S,
                                   int N, int H, int H_kv, int D, int L_cap, int max_prefix_len,
                                   float sm_scale, void *workspace, size_t workspace_bytes,
                                   int32_t *dev_status, hawk_stream_t stream);

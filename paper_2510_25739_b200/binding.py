@@ -180,7 +180,7 @@ def verify_attn(q: torch.Tensor, k_cache: torch.Tensor, v_cache: torch.Tensor, p
                 workspace: Optional[torch.Tensor] = None, dev_status: Optional[torch.Tensor] = None,
                 anc_mask: Optional[torch.Tensor] = None) -> torch.Tensor:
     """q [S,K,H,D], caches [S,H_kv,L_cap,D] (bf16), prefix_len [S] int32 -> out [S,K,H*D] bf16.
-    With anc_mask (int32 tensor holding the uint32 masks, [K]) the K rows are tree nodes (hawk_verify_attn_tree)."""
+    With anc_mask (int64 tensor holding the uint64 masks, [K]) the K rows are tree nodes (hawk_verify_attn_tree)."""
     lib = load_library()
     S, K, H, D = q.shape
     _, H_kv, L_cap, _ = k_cache.shape
@@ -196,7 +196,7 @@ def verify_attn(q: torch.Tensor, k_cache: torch.Tensor, v_cache: torch.Tensor, p
         workspace = torch.empty(need, dtype=torch.uint8, device=q.device)
     ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
     if anc_mask is not None:
-        _check(anc_mask, torch.int32, "anc_mask", (K,))
+        _check(anc_mask, torch.int64, "anc_mask", (K,))
         rc = lib.hawk_verify_attn_tree(_ptr(q), _ptr(k_cache), _ptr(v_cache), _ptr(prefix_len), _ptr(anc_mask),
                                        _ptr(out), S, K, H, H_kv, D, L_cap, int(max_prefix_len), float(sm_scale),
                                        _ptr(workspace), ws_bytes, _ptr(dev_status), _stream())

@@ -71,7 +71,7 @@ struct AttnParams {
     float *part;  // [workers][2 slots]{o[rows_per_item][D], (running max in log2 units, running sum)[rows_per_item]}
     int S, K, H, H_kv, L_cap;
     int pl_max;           // largest admissible prefix length: min(L_cap - K, max_prefix_len)
-    const uint32_t *anc_mask;  // [K] block rows visible to each query position; NULL: causal (row i sees rows <= i)
+    const uint64_t *anc_mask;  // [K] block rows visible to each query position; NULL: causal (row i sees rows <= i)
     int rows_per_item;    // query rows per item, a multiple of 8: the (head of the group, position) pairs of one
                           // kv head, numbered head-major, are cut into chunks of this many rows
     int chunks;           // items per kv head
@@ -145,11 +145,14 @@ __device__ __forceinline__ void step(Cursor &c, long long f_end, const AttnParam
 }
 
 // Is the key `rel` rows past the prefix visible to a query whose block-row mask is m?  Prefix keys
-// (rel < 0) always are; block rows past the 32nd never are.
-__device__ __forceinline__ bool key_visible(int rel, uint32_t m)
+// (rel < 0) always are; block rows past the 64th never are.
+__device__ __forceinline__ bool key_visible(int rel, uint64_t m)
 {
-    return rel < 0 || (rel < 32 && ((m >> rel) & 1u));
+    return rel < 0 || (rel < 64 && ((m >> rel) & 1ull));
 }
+
+// Mask of position `pos` of a plain chain: block rows 0 .. pos.
+__device__ __forceinline__ uint64_t chain_mask(int pos) { return pos >= 63 ? ~0ull : (2ull << pos) - 1ull; }
 
 __device__ __forceinline__ uint32_t movmatrix_trans(uint32_t x)
 {
@@ -257,7 +260,6 @@ __global__ void __launch_bounds__(kWarps * 32, kWarps == kWarpsGroup ? 3 : 1) at
     uint32_t qb[NQT][DB][2];  // Q^T as the 16 x 8 operand: query row = column tile * 8 + g
     float ot[NQT][DB][4];     // O^T accumulators
     float mrun[NQT][2], lrun[NQT][2];  // running max (log2 units) and this thread's share of the running sum
-    uint32_t qm[NQT][2];      // block rows visible to the queries in this thread's columns (bit m: row prefix + m)
     int cur_item = -1, hbase = 0, gr0 = 0, nrows = 0, seg_pl = 0, seg_s = 0;
     long long seg_start = 0;
 
@@ -385,8 +387,6 @@ __global__ void __launch_bounds__(kWarps * 32, kWarps == kWarpsGroup ? 3 : 1) at
                 for (int c = 0; c < 2; ++c) {
                     mrun[nq][c] = -CUDART_INF_F;
                     lrun[nq][c] = 0.f;
-                    const int pos = (gr0 + nq * 8 + 2 * tq + c) % P.K;  // (padding rows get some position's mask)
-                    qm[nq][c] = P.anc_mask ? P.anc_mask[pos] : (2u << pos) - 1u;
                 }
             }
         }
@@ -415,6 +415,16 @@ __global__ void __launch_bounds__(kWarps * 32, kWarps == kWarpsGroup ? 3 : 1) at
         }
         // ---- causal mask inside the block, which also hides the cache rows past the last visible key
         if (tile_key0 + TK > pl) {
+            // block rows visible to the queries in this thread's columns (bit m: row prefix + m); looked up here, at the
+            // few tiles of an item that reach into the block, rather than carried in registers through all the others
+            uint64_t qm[NQT][2];
+#pragma unroll
+            for (int nq = 0; nq < NQT; ++nq)
+#pragma unroll
+                for (int c = 0; c < 2; ++c) {
+                    const int pos = (gr0 + nq * 8 + 2 * tq + c) % P.K;  // (padding rows get some position's mask)
+                    qm[nq][c] = P.anc_mask ? P.anc_mask[pos] : chain_mask(pos);
+                }
 #pragma unroll
             for (int kb = 0; kb < KB; ++kb) {
                 const int rel0 = tile_key0 + kb * 16 + g - pl, rel1 = rel0 + 8;
@@ -877,7 +887,7 @@ cudaError_t launch_attn(const CUtensorMap &map_k, const CUtensorMap &map_v, cons
 
 extern "C" size_t hawk_verify_attn_workspace_bytes(int S, int K, int H, int H_kv, int D, int max_prefix_len)
 {
-    if (S <= 0 || K < 1 || K > 32 || H <= 0 || H_kv <= 0 || H % H_kv != 0 || (D != 64 && D != 128) ||
+    if (S <= 0 || K < 1 || K > 64 || H <= 0 || H_kv <= 0 || H % H_kv != 0 || (D != 64 && D != 128) ||
         max_prefix_len < 0)
         return 0;
     const AttnPlan pl = make_plan(S, K, H, H_kv, D, max_prefix_len);
@@ -893,7 +903,7 @@ hawk_status hawk_host::check_verify_attn_args(const void *q, const void *k_cache
     if (S < 0 || K < 0 || H < 0 || H_kv < 0 || D < 0 || L_cap < 0 || max_prefix_len < 0) return HAWK_ERR_SHAPE;
     if (S == 0) return HAWK_OK;
     if (!q || !k_cache || !v_cache || !prefix_len || !out) return HAWK_ERR_NULL;
-    if (K < 1 || K > 32 || (D != 64 && D != 128) || H < 1 || H_kv < 1 || H % H_kv != 0) return HAWK_ERR_UNSUPPORTED;
+    if (K < 1 || K > 64 || (D != 64 && D != 128) || H < 1 || H_kv < 1 || H % H_kv != 0) return HAWK_ERR_UNSUPPORTED;
     if (max_prefix_len + K > L_cap) return HAWK_ERR_SHAPE;
     if (static_cast<long long>(S) * H_kv * L_cap >= (1ll << 31)) return HAWK_ERR_UNSUPPORTED;
     if (!(sm_scale > 0.f) || isinf(sm_scale)) return HAWK_ERR_PARAM;
@@ -912,7 +922,7 @@ namespace {
 
 // Common body of hawk_verify_attn (anc_mask == NULL: causal block) and hawk_verify_attn_tree.
 hawk_status verify_attn_impl(const void *q, const void *k_cache, const void *v_cache, const int32_t *prefix_len,
-                             const uint32_t *anc_mask, void *out, int S, int K, int H, int H_kv, int D, int L_cap,
+                             const uint64_t *anc_mask, void *out, int S, int K, int H, int H_kv, int D, int L_cap,
                              int max_prefix_len, float sm_scale, void *workspace, size_t workspace_bytes,
                              int32_t *dev_status, hawk_stream_t stream)
 {
@@ -1010,7 +1020,7 @@ extern "C" hawk_status hawk_verify_attn(const void *q, const void *k_cache, cons
 }
 
 extern "C" hawk_status hawk_verify_attn_tree(const void *q, const void *k_cache, const void *v_cache,
-                                             const int32_t *prefix_len, const uint32_t *anc_mask, void *out, int S,
+                                             const int32_t *prefix_len, const uint64_t *anc_mask, void *out, int S,
                                              int N, int H, int H_kv, int D, int L_cap, int max_prefix_len,
                                              float sm_scale, void *workspace, size_t workspace_bytes,
                                              int32_t *dev_status, hawk_stream_t stream)

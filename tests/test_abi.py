@@ -84,7 +84,7 @@ def test_attn_argument_checks(lib):
     assert call(S=-1) == E_SHAPE
     assert call(q=None) == E_NULL
     assert call(out=None) == E_NULL
-    assert call(K=0) == E_UNSUP and call(K=33) == E_UNSUP
+    assert call(K=0) == E_UNSUP and call(K=65, L_cap=300) == E_UNSUP
     assert call(D=96) == E_UNSUP
     assert call(H=16, H_kv=3) == E_UNSUP
     assert call(mpl=129) == E_SHAPE                      # prefix + K exceeds the cache capacity
@@ -204,7 +204,7 @@ def test_attn_tree_argument_checks(lib):
     f = lib.hawk_verify_attn_tree
     assert f(p, p, p, p, None, p, 2, 7, 4, 4, 64, 100, 90, 0.125, None, 0, None, None) == E_NULL   # no mask
     assert f(p, p, p, p, p, p, 0, 7, 4, 4, 64, 100, 90, 0.125, None, 0, None, None) == OK
-    assert f(p, p, p, p, p, p, 2, 33, 4, 4, 64, 200, 90, 0.125, None, 0, None, None) == E_UNSUP
+    assert f(p, p, p, p, p, p, 2, 65, 4, 4, 64, 200, 90, 0.125, None, 0, None, None) == E_UNSUP
     assert f(p, p, p, p, p, p, 2, 22, 4, 4, 64, 100, 90, 0.125, None, 0, None, None) == E_SHAPE    # 90 + 22 > 100
 
 

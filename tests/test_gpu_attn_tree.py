@@ -32,7 +32,7 @@ def _check(branching, B, H, H_kv, D, L, seed, ragged=True, masks=None):
     status = torch.zeros(1, dtype=torch.int32, device="cuda")
     out = hawk.verify_attn(bf16_to_torch(a["q"]), bf16_to_torch(a["k_cache"]), bf16_to_torch(a["v_cache"]),
                            to_dev(a["prefix_len"]), int(a["prefix_len"].max()), float(a["sm_scale"]),
-                           dev_status=status, anc_mask=to_dev(masks.view(np.int32)))
+                           dev_status=status, anc_mask=to_dev(masks.view(np.int64)))
     torch.cuda.synchronize()
     assert int(status.item()) == 0
     got = torch_bf16_to_f64(out)
@@ -51,6 +51,11 @@ def _check(branching, B, H, H_kv, D, L, seed, ragged=True, masks=None):
     ((3, 3, 2), 1, 2, 2, 64, 1200),     # 31 nodes: four column tiles, keys split over several shares
     ((3, 2, 2), 1, 2, 2, 128, 200),     # 22 nodes at D = 128: two items of 16 and 6 rows per head
     ((2, 2), 1, 8, 2, 64, 150),         # grouped-query: 4 heads x 7 nodes share a kv head
+    ((3, 3, 3), 2, 2, 2, 64, 500),      # 40 nodes: mask bits past the 32nd, two items of 24 and 16 rows per head
+    ((4, 3, 2), 1, 2, 2, 128, 333),     # 41 nodes at D = 128: two items of 24 and 17 rows per head
+    ((2, 2, 2, 2, 2), 1, 3, 3, 64, 90), # 63 nodes
+    ((7, 8), 2, 2, 1, 64, 1100),        # 64 nodes, two query heads per kv head: four items of 32 rows
+    ((7, 8), 1, 2, 2, 128, 40),         # 64 nodes at D = 128: three items per head, the block longer than the prefix
 ])
 def test_tree_shapes(branching, B, H, H_kv, D, L):
     _check(branching, B, H, H_kv, D, L, seed=500 + L)
@@ -62,12 +67,30 @@ def test_chain_mask_is_the_causal_kernel_bit_for_bit():
     a = wl.make_attn_inputs(cfg, 3)
     args = (bf16_to_torch(a["q"]), bf16_to_torch(a["k_cache"]), bf16_to_torch(a["v_cache"]),
             to_dev(a["prefix_len"]), cfg.L, float(a["sm_scale"]))
-    masks = np.array([(2 << i) - 1 for i in range(cfg.K)], np.uint32)
+    masks = wl.chain_masks(cfg.K)
     o1 = hawk.verify_attn(*args)
-    o2 = hawk.verify_attn(*args, anc_mask=to_dev(masks.view(np.int32)))
+    o2 = hawk.verify_attn(*args, anc_mask=to_dev(masks.view(np.int64)))
     assert torch.equal(o1.view(torch.int16), o2.view(torch.int16))
 
 
 def test_config_shaped_tree():
     """22-node tree at the LlamaGen-XL shape (full-size launch, oracle on all of it: seconds)."""
     _check((3, 2, 2), 4, 20, 20, 64, 1144, seed=77, ragged=False)
+
+
+@pytest.mark.parametrize("K,D", [(33, 64), (48, 128), (64, 64)])
+def test_long_chains_against_the_causal_oracle(K, D):
+    """A plain chain of more than 32 drafts through hawk_verify_attn (no mask argument): the kernel's own chain
+    masks past the 32nd row, against the causal oracle."""
+    import paper_2510_25739_b200 as hawk
+    cfg = wl.config(1, B=1, K=K, H=2, H_kv=2, D=D, L=150)
+    a = wl.make_attn_inputs(cfg, 600 + K, ragged=True)
+    want = oracle.verify_attn(a["q"], a["k_cache"], a["v_cache"], a["prefix_len"], a["sm_scale"])
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    out = hawk.verify_attn(bf16_to_torch(a["q"]), bf16_to_torch(a["k_cache"]), bf16_to_torch(a["v_cache"]),
+                           to_dev(a["prefix_len"]), int(a["prefix_len"].max()), float(a["sm_scale"]), dev_status=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    got = torch_bf16_to_f64(out)
+    rms = np.sqrt((want ** 2).mean())
+    assert (np.abs(got - want) <= RTOL * np.abs(want) + ATOL_RMS * rms).all()
