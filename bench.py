@@ -897,12 +897,33 @@ def bench_e2e(cfg, reps, stream, torch, hawk, binding, world, dist, steps, warmu
             dist.barrier()
         torch.cuda.synchronize()
     ms = start.elapsed_time(stop)
+    # the floor of such a step on this machine: the same host buffers copied to the same device buffers, nothing else
+    with torch.cuda.stream(stream):
+        c0, c1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        n_copy = max(5, min(steps, 50))
+        pairs = [[(getattr(r, k), keep[j][0][k]) for k in ("q", "x", "q_probs", "draft", "u_accept", "u_resample")]
+                 for j, r in enumerate(reps)]
+        for dst, src in pairs[0]:
+            dst.copy_(src, non_blocking=True)
+        stream.synchronize()
+        c0.record(stream)
+        for it in range(n_copy):
+            for dst, src in pairs[it % n_rep]:
+                dst.copy_(src, non_blocking=True)
+        c1.record(stream)
+        stream.synchronize()
+    copy_ms = c0.elapsed_time(c1) / n_copy
     if dist is not None:
         t = torch.tensor([ms], device="cuda")
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
         ms = float(t.item())
     return {"value": cfg.B * cfg.K * world / (ms / steps * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
             "d2h_bytes_per_step": d2h, "ms_per_step": ms / steps, "steps": steps,
+            "h2d_GB/s": h2d / (ms / steps) / 1e6,
+            "copy_floor_ms_per_step": copy_ms, "copy_floor_GB/s": h2d / copy_ms / 1e6,
+            "step_over_copy_floor": (ms / steps) / copy_ms,
+            "bound": "the host-to-device copy of the draft distributions (q_probs is most of the step's host bytes); "
+                     "the kernels run under it on the caller's stream while it travels on the library's side stream",
             "api": "hawk_verify_step_host (pinned host inputs -> device, 3 kernels, results -> host)",
             "launch": mode}
 

@@ -57,6 +57,7 @@ typedef enum {
 #define HAWK_DEV_NONFINITE 4  /* a NaN or +inf logit was treated as -inf                        */
 #define HAWK_DEV_BAD_PREFIX 8 /* a prefix length lay outside [0, L_cap - K] and was clamped     */
 #define HAWK_DEV_BAD_TREE 16  /* a child range or draft-row index of the tree was out of range    */
+#define HAWK_DEV_BOUNDS 32    /* libraries built with -DHAWK_DEBUG only: an index lay outside its array, the access was skipped */
 
 const char *hawk_status_string(hawk_status status);
 int hawk_version(void); /* major*10000 + minor*100 + patch */
@@ -239,7 +240,12 @@ hawk_status hawk_tree_accept(const float *logits, const float *q_probs, const in
  *     lc = sum_c x[b*rows + i][c] * w[v][c],   lu = sum_c x[(B + b)*rows + i][c] * w[v][c]
  * for v_begin <= v < v_end: the accumulators of hawk_head_proj combined in fp32 by subtract, fused
  * multiply-add, divide (step 1 of hawk_cfg_accept, on the same numbers), so the two-call form decides
- * exactly as the three-call form does.
+ * exactly as the three-call form does wherever hawk_head_proj sums a logit in one chain.  The one
+ * exception: a hawk_head_proj call with few tiles and a long hidden dimension
+ * (2 * ceil((v_end - v_begin) / 128) <= SM count, M <= 256 and hidden >= 1024) sums each logit as two
+ * halves of the hidden dimension added together, which this call never does; there the two forms'
+ * logits agree within the tolerance stated for logits (each form against the exact sum), not bit for
+ * bit, and a decision that lies that close to its threshold can differ.
  *   x       bf16 [2B][rows][hidden]   conditional streams first, as everywhere
  *   w       bf16 [V][hidden]
  *   guided  fp32 [B][rows][V]         columns outside [v_begin, v_end) are not written

@@ -17,7 +17,7 @@ _PKG = Path(__file__).resolve().parent
 _LIB_PATH = _PKG / "libhawk_verify.so"
 _lib: Optional[ctypes.CDLL] = None
 
-DEV_TIMEOUT, DEV_BAD_DRAFT, DEV_NONFINITE, DEV_BAD_PREFIX, DEV_BAD_TREE = 1, 2, 4, 8, 16
+DEV_TIMEOUT, DEV_BAD_DRAFT, DEV_NONFINITE, DEV_BAD_PREFIX, DEV_BAD_TREE, DEV_BOUNDS = 1, 2, 4, 8, 16, 32
 
 EXPORTS = (
     "hawk_status_string", "hawk_version",

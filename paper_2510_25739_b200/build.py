@@ -94,5 +94,14 @@ def build_stall_variant(force: bool = False) -> Path:
                  extra_flags=("-DHAWK_WAIT_NS=2000000ull", "-DHAWK_TEST_STALL"))
 
 
+DEBUG_LIB = PKG / "libhawk_verify_debug.so"
+
+
+def build_debug_variant(force: bool = False) -> Path:
+    """The library with index checks compiled in (-DHAWK_DEBUG): every checked index that leaves its array raises
+    HAWK_DEV_BOUNDS in the call's status word and the access is skipped.  The stand-in for a memory checker."""
+    return build(force=force, lib=DEBUG_LIB, objdir=PKG / "_build_debug", extra_flags=("-DHAWK_DEBUG",))
+
+
 if __name__ == "__main__":
     print(build(force="--force" in sys.argv, verbose="-v" in sys.argv))

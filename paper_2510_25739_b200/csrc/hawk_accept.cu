@@ -178,6 +178,7 @@ struct RowShared {
     float wbase[VPT * (NT / 32)];
     int bin, above, tok, ncand;
     float tau, pxe, total;
+    int32_t *dbg_status;  // where the debug build's index checks report (set by the kernels; unused otherwise)
     int ctok[kMaxChildren];
     float cqx[kMaxChildren], cu[kMaxChildren];
 };
@@ -283,7 +284,7 @@ __device__ __forceinline__ float row_topk(const float (&x)[VPT][4], float mn, fl
                     const float v = x[j][c];
                     const bool in = v >= lo && v <= hi;
                     bins[j][c] = in ? min(kBins - 1, static_cast<int>((hi - v) * scale)) : -1;
-                    if (in) atomicAdd(&sh.hist[bins[j][c]], 1);
+                    if (in && HAWK_IN_BOUNDS(sh.dbg_status, bins[j][c], kBins)) atomicAdd(&sh.hist[bins[j][c]], 1);
                 }
             __syncthreads();
             int local = 0;
@@ -313,7 +314,10 @@ __device__ __forceinline__ float row_topk(const float (&x)[VPT][4], float mn, fl
                 for (int j = 0; j < VPT; ++j)
 #pragma unroll
                     for (int c = 0; c < 4; ++c)
-                        if (bins[j][c] == bstar) sh.cand[atomicAdd(&sh.ncand, 1)] = x[j][c];
+                        if (bins[j][c] == bstar) {
+                            const int at = atomicAdd(&sh.ncand, 1);
+                            if (HAWK_IN_BOUNDS(sh.dbg_status, at, kCandMax)) sh.cand[at] = x[j][c];
+                        }
                 __syncthreads();
                 if (C <= 32) {  // the usual case: one warp ranks them, all 32 exchanges in flight at once
                     if (warp == 0) {
@@ -497,6 +501,7 @@ __global__ void __launch_bounds__(NT) accept_rows_kernel(const AcceptParams P)
 {
     __shared__ RowShared<NT, VPT> sh;
     const int tid = threadIdx.x;
+    if (tid == 0) sh.dbg_status = P.dev_status;  // (published by the first block-wide barrier, long before its first use)
     hawk::allow_dependent_launch();
     hawk::grid_dependency_wait();
 
@@ -539,7 +544,7 @@ __global__ void __launch_bounds__(NT) accept_rows_kernel(const AcceptParams P)
             xd = xd < P.v_begin ? P.v_begin : P.v_begin + n - 1;
         }
         xd -= P.v_begin;
-        qx = qrow[xd];
+        if (HAWK_IN_BOUNDS(P.dev_status, xd, n)) qx = qrow[xd];
     }
     if (flags && P.dev_status) atomicOr(P.dev_status, flags);
 
@@ -550,7 +555,7 @@ __global__ void __launch_bounds__(NT) accept_rows_kernel(const AcceptParams P)
             float *pd = P.p_debug + (static_cast<size_t>(b) * P.rows + i) * P.V + P.v_begin;
             for (int e = tid; e < n; e += NT) pd[e] = 0.f;
         }
-        if (tid == 0) P.row_out[b * P.rows + i] = ROW_REJECTED_NO_TOKEN;
+        if (tid == 0 && HAWK_IN_BOUNDS(P.dev_status, b * P.rows + i, P.B * P.rows)) P.row_out[b * P.rows + i] = ROW_REJECTED_NO_TOKEN;
         return;
     }
 
@@ -576,7 +581,9 @@ __global__ void __launch_bounds__(NT) accept_rows_kernel(const AcceptParams P)
 #pragma unroll
             for (int c = 0; c < 4; ++c) {
                 const int e = 4 * (j * NT + tid) + c;
-                if (e < n) pd[e] = x[j][c] * invZ;
+                if (e < n && HAWK_IN_BOUNDS(P.dev_status, (static_cast<long long>(b) * P.rows + i) * P.V + P.v_begin + e,
+                                            static_cast<long long>(P.B) * P.rows * P.V))
+                    pd[e] = x[j][c] * invZ;
             }
     }
 
@@ -585,7 +592,7 @@ __global__ void __launch_bounds__(NT) accept_rows_kernel(const AcceptParams P)
         const float px = pxe * invZ;
         const bool accepted = static_cast<double>(u_acc) * static_cast<double>(qx) < static_cast<double>(px);
         if (accepted) {
-            if (tid == 0) P.row_out[b * P.rows + i] = ROW_ACCEPTED;
+            if (tid == 0 && HAWK_IN_BOUNDS(P.dev_status, b * P.rows + i, P.B * P.rows)) P.row_out[b * P.rows + i] = ROW_ACCEPTED;
             return;
         }
     }
@@ -615,7 +622,9 @@ __global__ void __launch_bounds__(NT) accept_rows_kernel(const AcceptParams P)
             continue;
         }
         const int tok = row_search<NT, VPT>(rr, sj, incl, u_res * total, sh);
-        if (tid == 0) P.row_out[b * P.rows + i] = tok >= 0 ? P.v_begin + tok : ROW_REJECTED_NO_TOKEN;
+        if (tid == 0 && HAWK_IN_BOUNDS(P.dev_status, b * P.rows + i, P.B * P.rows) &&
+            (tok == -1 || HAWK_IN_BOUNDS(P.dev_status, tok, n)))
+            P.row_out[b * P.rows + i] = tok >= 0 ? P.v_begin + tok : ROW_REJECTED_NO_TOKEN;
         return;
     }
 }
@@ -653,6 +662,7 @@ __global__ void __launch_bounds__(NT) tree_rows_kernel(const TreeParams P)
     __shared__ RowShared<NT, VPT> sh;
     __shared__ int s_cq[kMaxChildren];
     const int tid = threadIdx.x;
+    if (tid == 0) sh.dbg_status = P.dev_status;
     hawk::allow_dependent_launch();
     hawk::grid_dependency_wait();
 
@@ -719,7 +729,8 @@ __global__ void __launch_bounds__(NT) tree_rows_kernel(const TreeParams P)
             flags |= HAWK_DEV_BAD_TREE;
             my_q = max(0, min(my_q, P.NQ - 1));
         }
-        my_qx = P.q[(static_cast<size_t>(b) * P.NQ + my_q) * P.V + P.v_begin + my_tok];
+        if (HAWK_IN_BOUNDS(P.dev_status, my_tok, n) && HAWK_IN_BOUNDS(P.dev_status, my_q, P.NQ))
+            my_qx = P.q[(static_cast<size_t>(b) * P.NQ + my_q) * P.V + P.v_begin + my_tok];
     }
     if (flags && P.dev_status) atomicOr(P.dev_status, flags);
 
@@ -751,7 +762,8 @@ __global__ void __launch_bounds__(NT) tree_rows_kernel(const TreeParams P)
         const float px = sh.pxe / mass;
         const bool accepted = static_cast<double>(sh.cu[ci]) * static_cast<double>(sh.cqx[ci]) < static_cast<double>(px);
         if (accepted) {
-            if (tid == 0) P.verdict[b * P.N + node] = cb + ci;
+            if (tid == 0 && HAWK_IN_BOUNDS(P.dev_status, b * P.N + node, P.B * P.N) && HAWK_IN_BOUNDS(P.dev_status, cb + ci, P.N))
+                P.verdict[b * P.N + node] = cb + ci;
             return;
         }
         // rejected: target <- max(0, p - q), kept un-normalised as max(0, x - mass * q)
@@ -788,7 +800,7 @@ __global__ void __launch_bounds__(NT) tree_rows_kernel(const TreeParams P)
     const float total = row_mass<NT, VPT>(x, sj, incl, sh);
     int tok = -1;
     if (total > 0.f) tok = row_search<NT, VPT>(x, sj, incl, u_res * total, sh);
-    if (tid == 0) P.verdict[b * P.N + node] = tok >= 0 ? -(P.v_begin + tok) - 2 : -1;
+    if (tid == 0 && HAWK_IN_BOUNDS(P.dev_status, b * P.N + node, P.B * P.N)) P.verdict[b * P.N + node] = tok >= 0 ? -(P.v_begin + tok) - 2 : -1;
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -802,6 +814,7 @@ __global__ void __launch_bounds__(NT) pool_sample_kernel(const float *pool_q, co
 {
     __shared__ RowShared<NT, VPT> sh;
     const int tid = threadIdx.x;
+    if (tid == 0) sh.dbg_status = dev_status;
     hawk::allow_dependent_launch();
     hawk::grid_dependency_wait();
     const float *qrow = pool_q + static_cast<size_t>(blockIdx.x) * V + v_begin;
@@ -831,7 +844,8 @@ __global__ void __launch_bounds__(NT) pool_sample_kernel(const float *pool_q, co
         }
         const int want = node_q[node];
         bad |= (want < 0 || want >= NQ) ? 1 : 0;
-        if (max(0, min(want, NQ - 1)) == r) node_token[b * N + node] = token;
+        if (max(0, min(want, NQ - 1)) == r && (token == -1 || HAWK_IN_BOUNDS(dev_status, token - v_begin, n)))
+            node_token[b * N + node] = token;
     }
     if (bad && dev_status) atomicOr(dev_status, HAWK_DEV_BAD_TREE);
 }
@@ -874,7 +888,7 @@ __global__ void tree_walk_kernel(const int32_t *verdict, int B, int N, int max_d
             if (dev_status) atomicOr(dev_status, HAWK_DEV_BAD_TREE);
             break;
         }
-        if (path && depth < max_depth) path[b * max_depth + depth] = v;
+        if (path && depth < max_depth && HAWK_IN_BOUNDS(dev_status, b * max_depth + depth, B * max_depth)) path[b * max_depth + depth] = v;
         ++depth;
         node = v;
     }

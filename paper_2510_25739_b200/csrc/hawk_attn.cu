@@ -291,7 +291,8 @@ __global__ void __launch_bounds__(kWarps * 32, kWarps == kWarpsGroup ? 3 : 1) at
                     // (dims g / g+8) x (queries 2tq, 2tq+1)  ->  (query g) x (dims 2tq, 2tq+1 / +8)
                     const uint32_t lo = movmatrix_trans(pack_bf16(ot[nq][db][0] * inv0, ot[nq][db][1] * inv1));
                     const uint32_t hi = movmatrix_trans(pack_bf16(ot[nq][db][2] * inv0, ot[nq][db][3] * inv1));
-                    if (valid) {
+                    if (valid && HAWK_IN_BOUNDS(P.dev_status, (dst - P.out) + db * 16 + 9,
+                                                static_cast<long long>(P.S) * P.K * P.H * D)) {
                         *reinterpret_cast<uint32_t *>(dst + db * 16) = lo;
                         *reinterpret_cast<uint32_t *>(dst + db * 16 + 8) = hi;
                     }
@@ -303,6 +304,11 @@ __global__ void __launch_bounds__(kWarps * 32, kWarps == kWarpsGroup ? 3 : 1) at
             float *ps = grouped ? reinterpret_cast<float *>(ring)
                                 : P.part + (static_cast<size_t>(w) * 2 + slot) * P.rows_per_item * (D + 2);
             if (grouped && lane == 0) has_part[warp] = 1;
+            // (debug build: a partial must fit the warp's ring, or its slot of the workspace)
+            if (!HAWK_IN_BOUNDS(P.dev_status, P.rows_per_item * (D + 2) * 4 - 1,
+                                grouped ? kStages * kStageBytes : P.rows_per_item * (D + 2) * 4) ||
+                !HAWK_IN_BOUNDS(P.dev_status, grouped ? 0 : w * 2 + slot, grouped ? 1 : P.workers * 2))
+                return;
 #pragma unroll
             for (int nq = 0; nq < NQT; ++nq)
 #pragma unroll
@@ -396,6 +402,10 @@ __global__ void __launch_bounds__(kWarps * 32, kWarps == kWarpsGroup ? 3 : 1) at
 
         ok = mbar_wait(&full_bar[st], ph, nullptr);
         if (!ok) break;
+        // (debug build: the tile's rows lie inside the cache and the stage inside the warp's ring)
+        if (!HAWK_IN_BOUNDS(P.dev_status, cc.row_base + tile_key0, static_cast<long long>(P.S) * P.H_kv * P.L_cap) ||
+            !HAWK_IN_BOUNDS(P.dev_status, st, kStages))
+            break;
         const uint32_t kbase = ring_u32 + st * kStageBytes;
         const uint32_t vbase = kbase + C::kHalves * C::kSubTileBytes;
 
@@ -830,7 +840,10 @@ AttnPlan make_plan(int S, int K, int H, int H_kv, int D, int max_prefix_len)
     pl.group_g = 0;
     // (with fewer than 222 items the 4 warps per item are fewer than three quarters of the shares' 1184 workers:
     // long items then go faster as shares)
-    if (pl.rows_per_item == 8 && 4 * pl.items >= 3 * kPlanSms * 2 && pl.items <= 3 * kPlanSms &&
+#ifndef HAWK_ATTN_GROUP_MAX_ROWS
+#define HAWK_ATTN_GROUP_MAX_ROWS 8
+#endif
+    if (pl.rows_per_item <= HAWK_ATTN_GROUP_MAX_ROWS && 4 * pl.items >= 3 * kPlanSms * 2 && pl.items <= 3 * kPlanSms &&
         pl.tiles_per_item >= 2 * kWarpsGroup) {
         pl.group_g = kWarpsGroup;
         pl.whole = false;  // (from 8 tiles on, four warps with a merge in shared memory beat one warp alone)

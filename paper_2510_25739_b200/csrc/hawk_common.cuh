@@ -28,6 +28,21 @@ constexpr uint32_t kTestStallBytes = 16;
 constexpr uint32_t kTestStallBytes = 0;
 #endif
 
+// Index checks of the debug build (-DHAWK_DEBUG; the stand-in for a memory checker, which cannot be run here):
+// HAWK_IN_BOUNDS(status, i, n) is true when 0 <= i < n; otherwise it raises HAWK_DEV_BOUNDS in *status (if not
+// NULL) and yields false, and the caller skips the access.  In regular builds it is the constant true.
+#ifdef HAWK_DEBUG
+__device__ __forceinline__ bool in_bounds(int32_t *status, long long i, long long n)
+{
+    if (i >= 0 && i < n) return true;
+    if (status) atomicOr(status, HAWK_DEV_BOUNDS);
+    return false;
+}
+#define HAWK_IN_BOUNDS(status, i, n) (::hawk::in_bounds((status), static_cast<long long>(i), static_cast<long long>(n)))
+#else
+#define HAWK_IN_BOUNDS(status, i, n) (true)
+#endif
+
 __device__ __forceinline__ uint32_t smem_u32(const void *p)
 {
     return static_cast<uint32_t>(__cvta_generic_to_shared(p));

@@ -75,7 +75,7 @@ __device__ __forceinline__ void epilogue_store(const HeadParams &P, uint32_t tad
 #pragma unroll
                 for (int j = 0; j < 16; ++j) {
                     const int n = nbase + j;
-                    if (n < P.M) {
+                    if (n < P.M && HAWK_IN_BOUNDS(P.dev_status, v, P.V)) {
                         float *dst = &P.logits[static_cast<size_t>(n) * P.V + v];
                         if constexpr (KSPLIT) atomicAdd(dst, __uint_as_float(r[j]));  // two addends onto zero: any order
                         else *dst = __uint_as_float(r[j]);
@@ -106,7 +106,7 @@ __device__ __forceinline__ void epilogue_store(const HeadParams &P, uint32_t tad
                     const float lc = __uint_as_float(rc[j]), lu = __uint_as_float(ru[j]);
                     float g = __fmaf_rn(P.cfg_scale, __fsub_rn(lc, lu), lu);
                     if (!unit_T) g = __fdiv_rn(g, P.temperature);
-                    if (pair < P.pairs) P.logits[static_cast<size_t>(pair) * P.V + v] = g;
+                    if (pair < P.pairs && HAWK_IN_BOUNDS(P.dev_status, v, P.V)) P.logits[static_cast<size_t>(pair) * P.V + v] = g;
                 }
             }
         }

@@ -47,6 +47,7 @@ __global__ void cache_put_kernel(const float *q_vert, const int32_t *position, f
     const int pos = position[b];
     if (pos < 0) return;
     const int slot = cache_slot(IW, VSD, pos, d);
+    if (!HAWK_IN_BOUNDS(nullptr, slot, slots)) return;  // (debug build; these kernels have no status word: the copy is skipped)
     copy_row(rows + (static_cast<size_t>(b) * slots + slot) * V, q_vert + (static_cast<size_t>(b) * VSD + d - 1) * V, V,
              vec != 0);
     if (blockIdx.y == 0 && threadIdx.x == 0) tags[b * slots + slot] = pos;
@@ -70,7 +71,7 @@ __global__ void pool_build_kernel(const float *q_horiz, const float *rows, const
         source = -j;  // missing until found
         if (position[b] >= 0 && from >= 0) {
             const int slot = cache_slot(IW, VSD, from, j);
-            if (tags[b * slots + slot] == from) {
+            if (HAWK_IN_BOUNDS(nullptr, slot, slots) && tags[b * slots + slot] == from) {
                 src = rows + (static_cast<size_t>(b) * slots + slot) * V;
                 source = j;
             }
