@@ -598,6 +598,10 @@ __global__ void __launch_bounds__(NT) accept_rows_kernel(const AcceptParams P)
     }
 
     // ---- rejected (or bonus row): inverse-CDF draw from max(0, p - q), or from p itself
+    // The rejection itself is published at once (the token follows): rows of later positions that start while this
+    // block is still drawing its token see that their chain has ended and do nothing.
+    if (P.skip_mode && !bonus && tid == 0)
+        *reinterpret_cast<volatile int32_t *>(&P.row_out[b * P.rows + i]) = ROW_REJECTED_NO_TOKEN;
     bool use_q = !bonus;
     for (int attempt = 0; attempt < 2; ++attempt) {
         float rr[VPT][4], sj[VPT], incl[VPT];  // residual weights of this thread's ids and their running sums
@@ -796,6 +800,9 @@ __global__ void __launch_bounds__(NT) tree_rows_kernel(const TreeParams P)
     }
 
     // ---- every candidate rejected (or a leaf): draw the correction token from the target as refined
+    // (the outcome "no child was picked" is published at once, the token follows: the children's blocks that start
+    // in the meantime see that the walk cannot reach them)
+    if (P.skip_mode && nc > 0 && tid == 0) *reinterpret_cast<volatile int32_t *>(&P.verdict[b * P.N + node]) = -1;
     float sj[VPT], incl[VPT];
     const float total = row_mass<NT, VPT>(x, sj, incl, sh);
     int tok = -1;
@@ -1025,7 +1032,10 @@ hawk_status cfg_accept_impl(const float *logits, int guided_in, const float *q_p
     // more rows than SMs: the later rows can see the verdicts of the earlier ones (see accept_rows_kernel)
     int sm_count = 0;
     (void)hawk_host::is_sm100(&sm_count);
-    P.skip_mode = (grid > sm_count + sm_count / 2 && !p_debug) ? 1 : 0;  // below 1.5 waves the marking costs more than it saves
+#ifndef HAWK_ACCEPT_SKIP_WAVES_X4
+#define HAWK_ACCEPT_SKIP_WAVES_X4 6  // quarter waves of rows from which verdicts are marked and looked at: 6 = 1.5 waves
+#endif
+    P.skip_mode = (4 * grid > HAWK_ACCEPT_SKIP_WAVES_X4 * sm_count && !p_debug) ? 1 : 0;
     if (P.skip_mode) {
         err = hawk_host::launch_dependent(accept_clear_kernel, dim3((grid + 255) / 256), dim3(256), 0, st, P.row_out, grid);
         if (err != cudaSuccess) return HAWK_ERR_CUDA;
