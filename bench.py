@@ -355,13 +355,10 @@ ACCEPT_TRAFFIC_BYTES = {2: 6_066_000, 4: 1_877_000, 5: 35_575_000}
 
 
 def launches_per_step(cfg, first, sms):
-    """Kernels one verify step launches: attention (+ its merge kernel when items are cut), head (+ a zeroing
-    kernel when its tiles are split along the hidden dimension), accept rows + per-sequence pass (+ a marking
-    kernel from 1.5 waves of rows on)."""
-    head_tiles = -(-cfg.V_valid // 128) * -(-cfg.M // 256)
-    head_split = cfg.M < 512 and 2 * head_tiles <= sms and cfg.hidden // 64 >= 16
+    """Kernels one verify step launches: attention (+ its merge kernel when items are cut), head, accept rows +
+    per-sequence pass (+ a marking kernel from 1.5 waves of rows on)."""
     accept_marks = cfg.B * cfg.K > sms + sms // 2
-    return (2 if first.attn_split else 1) + (2 if head_split else 1) + (3 if accept_marks else 2)
+    return (2 if first.attn_split else 1) + 1 + (3 if accept_marks else 2)
 
 
 def run_config(cid, args, torch, hawk, binding, world, rank, local_rank, dist, headline):

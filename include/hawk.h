@@ -240,12 +240,8 @@ hawk_status hawk_tree_accept(const float *logits, const float *q_probs, const in
  *     lc = sum_c x[b*rows + i][c] * w[v][c],   lu = sum_c x[(B + b)*rows + i][c] * w[v][c]
  * for v_begin <= v < v_end: the accumulators of hawk_head_proj combined in fp32 by subtract, fused
  * multiply-add, divide (step 1 of hawk_cfg_accept, on the same numbers), so the two-call form decides
- * exactly as the three-call form does wherever hawk_head_proj sums a logit in one chain.  The one
- * exception: a hawk_head_proj call with few tiles and a long hidden dimension
- * (2 * ceil((v_end - v_begin) / 128) <= SM count, M <= 256 and hidden >= 1024) sums each logit as two
- * halves of the hidden dimension added together, which this call never does; there the two forms'
- * logits agree within the tolerance stated for logits (each form against the exact sum), not bit for
- * bit, and a decision that lies that close to its threshold can differ.
+ * exactly as the three-call form does.  (Where a call has few tiles and a long hidden dimension, both
+ * hawk_head_proj and this call sum each logit as two halves of the hidden dimension, in the same way.)
  *   x       bf16 [2B][rows][hidden]   conditional streams first, as everywhere
  *   w       bf16 [V][hidden]
  *   guided  fp32 [B][rows][V]         columns outside [v_begin, v_end) are not written

@@ -42,7 +42,8 @@ struct HeadParams {
     int stages;
     int stage_bytes;
     int wide;      // pair kernel: one accumulator of BN (up to 512) columns, every k-step as two MMAs of BN / 2 columns
-    int ksplit;    // 1, or 2: two work units per tile, each over half of the hidden dimension (output zeroed first)
+    int ksplit;    // 1, or 2: a pair of blocks per tile, each over half of the hidden dimension; block 1 hands its sums to block 0
+    int xchg_off;  // ksplit == 2: byte offset, in a block's shared memory, of the buffer that receives the partner's sums
     int pairs;     // 0: plain logits; > 0: guided logits of this many (sequence, position) pairs
     float cfg_scale, temperature;
     int32_t *dev_status;
@@ -55,9 +56,27 @@ struct HeadParams {
 // WIDE (pair kernel, two MMAs of BN / 2 columns per k-step): accumulator column t of MMA half c = t / (BN / 2)
 // comes from CTA (t % (BN / 2)) / (BN / 4), row c * (BN / 4) + t % (BN / 4) of that CTA's token rows; BN is a
 // multiple of 64 there, so a 16-column chunk never straddles two of these ranges.
+// r += the partner block's sums for 16-column chunk `col / 16` of accumulator row `row` (own + partner, in that order).
+__device__ __forceinline__ void add_partner(uint32_t (&r)[16], const float *partner, int col, int row)
+{
+    const float4 *src = reinterpret_cast<const float4 *>(partner + (static_cast<size_t>(col >> 4) * kBM + row) * 16);
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+        const float4 a = src[q];
+        r[4 * q + 0] = __float_as_uint(__fadd_rn(__uint_as_float(r[4 * q + 0]), a.x));
+        r[4 * q + 1] = __float_as_uint(__fadd_rn(__uint_as_float(r[4 * q + 1]), a.y));
+        r[4 * q + 2] = __float_as_uint(__fadd_rn(__uint_as_float(r[4 * q + 2]), a.z));
+        r[4 * q + 3] = __float_as_uint(__fadd_rn(__uint_as_float(r[4 * q + 3]), a.w));
+    }
+}
+
+// KSPLIT: `partner` holds the other block's sums over its half of the hidden dimension, 16-column chunk k of
+// accumulator row `row` at partner[(k * 128 + row) * 16 ..]; they are added to this block's (this + partner, always
+// in that order) before anything else happens to the value.
 template <bool KSPLIT = false, bool WIDE = false>
 __device__ __forceinline__ void epilogue_store(const HeadParams &P, uint32_t taddr, int tn, int v, bool v_ok,
-                                               int chunk0 = 0, int chunk_step = 1)
+                                               int chunk0 = 0, int chunk_step = 1, const float *partner = nullptr,
+                                               int row = 0)
 {
     if (P.pairs == 0) {
         const int n0 = tn * P.BN;
@@ -65,6 +84,7 @@ __device__ __forceinline__ void epilogue_store(const HeadParams &P, uint32_t tad
             uint32_t r[16];
             tmem_ld_32x16(taddr + c, r);
             tmem_ld_wait();
+            if constexpr (KSPLIT) add_partner(r, partner, c, row);
             int nbase = n0 + c;
             if constexpr (WIDE) {
                 const int half = P.BN / 2, quarter = P.BN / 4;
@@ -77,8 +97,7 @@ __device__ __forceinline__ void epilogue_store(const HeadParams &P, uint32_t tad
                     const int n = nbase + j;
                     if (n < P.M && HAWK_IN_BOUNDS(P.dev_status, v, P.V)) {
                         float *dst = &P.logits[static_cast<size_t>(n) * P.V + v];
-                        if constexpr (KSPLIT) atomicAdd(dst, __uint_as_float(r[j]));  // two addends onto zero: any order
-                        else *dst = __uint_as_float(r[j]);
+                        *dst = __uint_as_float(r[j]);
                     }
                 }
             }
@@ -99,6 +118,10 @@ __device__ __forceinline__ void epilogue_store(const HeadParams &P, uint32_t tad
             tmem_ld_32x16(taddr + col_c, rc);
             tmem_ld_32x16(taddr + col_u, ru);
             tmem_ld_wait();
+            if constexpr (KSPLIT) {
+                add_partner(rc, partner, col_c, row);
+                add_partner(ru, partner, col_u, row);
+            }
             if (v_ok) {
 #pragma unroll
                 for (int j = 0; j < 16; ++j) {
@@ -113,8 +136,28 @@ __device__ __forceinline__ void epilogue_store(const HeadParams &P, uint32_t tad
     }
 }
 
-// KSPLIT: a unit of work is half of a tile's k-blocks and the halves add their results (see head_proj_impl).
-template <bool KSPLIT>
+// A block of a pair hands the accumulator chunks that its partner will finish (this thread's row of them) to the
+// partner's exchange buffer.  Ownership alternates by 16-column chunk: plain logits, chunk k belongs to block k % 2;
+// guided logits, the chunks of pairs 16k .. 16k + 15 (their conditional and their unconditional columns) to block k % 2.
+__device__ __forceinline__ void epilogue_send(const HeadParams &P, uint32_t taddr, int row, uint32_t partner_buf, int partner)
+{
+    const int half = P.BN / 2;
+    for (int c = 0; c < P.BN; c += 16) {
+        const int owner = ((P.pairs == 0 ? c : c % half) >> 4) & 1;
+        if (owner != partner) continue;
+        uint32_t r[16];
+        tmem_ld_32x16(taddr + c, r);
+        tmem_ld_wait();
+        const uint32_t dst = partner_buf + static_cast<uint32_t>(((c >> 4) * kBM + row) * 64);
+#pragma unroll
+        for (int q = 0; q < 4; ++q)
+            asm volatile("st.shared::cluster.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst + 16 * q), "r"(r[4 * q]), "r"(r[4 * q + 1]),
+                         "r"(r[4 * q + 2]), "r"(r[4 * q + 3])
+                         : "memory");
+    }
+}
+
+// One block per tile of 128 token ids x BN token rows, persistent over the tiles.
 __global__ void __launch_bounds__(kHeadThreads, 1) head_proj_kernel(const __grid_constant__ CUtensorMap map_w,
                                                                     const __grid_constant__ CUtensorMap map_x,
                                                                     const HeadParams P)
@@ -131,10 +174,7 @@ __global__ void __launch_bounds__(kHeadThreads, 1) head_proj_kernel(const __grid
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     hawk::allow_dependent_launch();
     const int kblocks = P.hidden / kBK;
-    // a unit of work is a tile, or (ksplit == 2) one half of a tile's k-blocks; the halves add their results
-    constexpr int kSplit = KSPLIT ? 2 : 1;
-    const int total_tiles = P.tiles_m * P.tiles_n * kSplit;
-    const int kb_half = (kblocks + kSplit - 1) / kSplit;
+    const int total_tiles = P.tiles_m * P.tiles_n;
 
     if (tid == 0) {
         for (int i = 0; i < P.stages; ++i) {
@@ -169,11 +209,9 @@ __global__ void __launch_bounds__(kHeadThreads, 1) head_proj_kernel(const __grid
             bool ok = true;
             long long issued = 0;
             for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
-                const int part = tile % kSplit, t2 = tile / kSplit;
-                const int tn = t2 % P.tiles_n, tm = t2 / P.tiles_n;
+                const int tn = tile % P.tiles_n, tm = tile / P.tiles_n;
                 const int row_w = P.v_begin + tm * kBM, row_x = tn * P.BN;
-                const int kb0 = part * kb_half, kb1 = min(kblocks, kb0 + kb_half);
-                for (int kb = kb0; kb < kb1; ++kb) {
+                for (int kb = 0; kb < kblocks; ++kb) {
                     ok = mbar_wait(&empty_bar[st], ph ^ 1u, abort_flag);
                     if (!ok) break;
                     uint8_t *a = smem + static_cast<size_t>(st) * P.stage_bytes;
@@ -216,7 +254,177 @@ __global__ void __launch_bounds__(kHeadThreads, 1) head_proj_kernel(const __grid
                 if (!ok) break;
                 tcgen05_fence_after();
                 const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(ab * P.BN);
-                const int part = tile % kSplit;
+                for (int kb = 0; kb < kblocks; ++kb) {
+                    ok = mbar_wait(&full_bar[st], ph, abort_flag);
+                    if (!ok) break;
+                    tcgen05_fence_after();
+                    const uint32_t a_addr = smem_u32(smem + static_cast<size_t>(st) * P.stage_bytes);
+                    const uint64_t da = umma_desc_k_major_sw128(a_addr);
+                    const uint64_t db = umma_desc_k_major_sw128(a_addr + kATileBytes);
+#pragma unroll
+                    for (int k = 0; k < kBK / 16; ++k) {
+                        // 16 bf16 along K = 32 bytes = 2 units of the descriptor's 16-byte address field
+                        umma_bf16(d_tmem, da + static_cast<uint64_t>(2 * k), db + static_cast<uint64_t>(2 * k), idesc,
+                                  (kb | k) != 0 ? 1u : 0u);
+                    }
+                    umma_commit(&empty_bar[st]);  // stage reusable once these MMAs have read it
+                    if (++st == P.stages) {
+                        st = 0;
+                        ph ^= 1u;
+                    }
+                }
+                if (!ok) break;
+                umma_commit(&acc_full[ab]);  // accumulator complete
+            }
+            if (!ok) {
+                *abort_flag = 1;
+                if (P.dev_status) atomicOr(P.dev_status, HAWK_DEV_TIMEOUT);
+            }
+        }
+    } else {
+        // =========================== epilogue warps: TMEM lanes 32*(warp%4) .. +31
+        const int lane_base = (warp & 3) * 32;
+        bool ok = true;
+        int it = 0;
+        for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++it) {
+            const int tn = tile % P.tiles_n, tm = tile / P.tiles_n;
+            const int ab = it & 1;
+            const uint32_t acc_ph = (it >> 1) & 1;
+            ok = mbar_wait(&acc_full[ab], acc_ph, abort_flag);
+            if (!ok) break;
+            tcgen05_fence_after();
+            const int v = P.v_begin + tm * kBM + lane_base + lane;  // this thread's token id
+            const bool v_ok = v < P.v_end;
+            const uint32_t taddr = tmem_base + (static_cast<uint32_t>(lane_base) << 16) + static_cast<uint32_t>(ab * P.BN);
+            epilogue_store(P, taddr, tn, v, v_ok);
+            tcgen05_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&acc_empty[ab]);
+        }
+        if (!ok && lane == 0) {
+            *abort_flag = 1;
+            if (P.dev_status) atomicOr(P.dev_status, HAWK_DEV_TIMEOUT);
+        }
+    }
+
+    tcgen05_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tcgen05_fence_after();
+        tmem_dealloc(tmem_base, kTmemCols);
+    }
+}
+
+
+
+// Few tiles and a long hidden dimension: launched as clusters of two blocks, one tile per cluster: block r multiplies over half r of the hidden
+// dimension; the blocks then swap halves of their accumulators through distributed shared memory (16-column chunks
+// alternate between them), each adds its partner's sums to its own for the chunks it owns (one addition of two
+// numbers: the result does not depend on timing or on which block does it), applies the guidance combine if asked to,
+// and stores.  No zeroed output, no atomics, and the plain and the guided form sum in the same way.
+__global__ void __launch_bounds__(kHeadThreads, 1) head_proj_split_kernel(const __grid_constant__ CUtensorMap map_w,
+                                                                    const __grid_constant__ CUtensorMap map_x,
+                                                                    const HeadParams P)
+{
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    uint64_t *full_bar = reinterpret_cast<uint64_t *>(smem + static_cast<size_t>(P.stages) * P.stage_bytes);
+    uint64_t *empty_bar = full_bar + kMaxStages;
+    uint64_t *acc_full = empty_bar + kMaxStages;  // [2]
+    uint64_t *acc_empty = acc_full + 2;           // [2]
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(acc_empty + 2);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    hawk::allow_dependent_launch();
+    const int kblocks = P.hidden / kBK;
+    // a block's unit of work is the half of its pair's tile that its rank in the pair names (the launch gives every
+    // pair exactly one tile; the loops below are written like the unsplit kernel's and run once)
+    const int total_tiles = P.tiles_m * P.tiles_n;
+    const int kb_half = (kblocks + 1) / 2;
+    const int part = static_cast<int>(cluster_cta_rank());
+    const int first_tile = static_cast<int>(blockIdx.x >> 1);
+    const int tile_step = static_cast<int>(gridDim.x >> 1);
+
+    if (tid == 0) {
+        for (int i = 0; i < P.stages; ++i) {
+            mbar_init(&full_bar[i], 1);
+            mbar_init(&empty_bar[i], 1);
+        }
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(&acc_full[i], 1);
+            mbar_init(&acc_empty[i], 4);  // one arrival per epilogue warp
+        }
+        *abort_flag = 0;
+        fence_mbar_init();
+    }
+    if (warp == 1) {
+        tmem_alloc(tmem_slot, kTmemCols);
+        tmem_relinquish();
+    }
+    tcgen05_fence_before();
+    __syncthreads();
+    tcgen05_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+    grid_dependency_wait();  // set-up above overlaps the previous kernel; global memory is touched from here on
+
+    if (warp == 0) {
+        // =========================== TMA producer
+        if (lane == 0) {
+            prefetch_tensormap(&map_w);
+            prefetch_tensormap(&map_x);
+            const uint32_t tx_bytes = static_cast<uint32_t>(P.stage_bytes);
+            int st = 0;
+            uint32_t ph = 0;
+            bool ok = true;
+            long long issued = 0;
+            for (int tile = first_tile; tile < total_tiles && ok; tile += tile_step) {
+                const int tn = tile % P.tiles_n, tm = tile / P.tiles_n;
+                const int row_w = P.v_begin + tm * kBM, row_x = tn * P.BN;
+                const int kb0 = part * kb_half, kb1 = min(kblocks, kb0 + kb_half);
+                for (int kb = kb0; kb < kb1; ++kb) {
+                    ok = mbar_wait(&empty_bar[st], ph ^ 1u, abort_flag);
+                    if (!ok) break;
+                    uint8_t *a = smem + static_cast<size_t>(st) * P.stage_bytes;
+                    // (test builds only: the first stage of block 0 is armed for more bytes than arrive)
+                    const bool stall = kTestStallBytes != 0 && blockIdx.x == 0 && issued == 0;
+                    mbar_arrive_expect_tx(&full_bar[st], tx_bytes + (stall ? kTestStallBytes : 0u));
+                    tma_load_2d(a, &map_w, kb * kBK, row_w, &full_bar[st]);
+                    if (P.pairs == 0) {
+                        tma_load_2d(a + kATileBytes, &map_x, kb * kBK, row_x, &full_bar[st]);
+                    } else {  // conditional rows of the tile's pairs, then their unconditional rows
+                        const int half = P.BN / 2;
+                        tma_load_2d(a + kATileBytes, &map_x, kb * kBK, tn * half, &full_bar[st]);
+                        tma_load_2d(a + kATileBytes + half * kBK * 2, &map_x, kb * kBK, P.pairs + tn * half,
+                                    &full_bar[st]);
+                    }
+                    ++issued;
+                    if (++st == P.stages) {
+                        st = 0;
+                        ph ^= 1u;
+                    }
+                }
+            }
+            if (!ok) {
+                *abort_flag = 1;
+                if (P.dev_status) atomicOr(P.dev_status, HAWK_DEV_TIMEOUT);
+            }
+        }
+    } else if (warp == 1) {
+        // =========================== MMA issuer
+        if (lane == 0) {
+            const uint32_t idesc = umma_idesc_bf16_f32(kBM, P.BN);
+            int st = 0;
+            uint32_t ph = 0;
+            bool ok = true;
+            int it = 0;
+            for (int tile = first_tile; tile < total_tiles && ok; tile += tile_step, ++it) {
+                const int ab = it & 1;
+                const uint32_t acc_ph = (it >> 1) & 1;
+                ok = mbar_wait(&acc_empty[ab], acc_ph ^ 1u, abort_flag);  // epilogue drained this buffer
+                if (!ok) break;
+                tcgen05_fence_after();
+                const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(ab * P.BN);
                 const int kb0 = part * kb_half, kb1 = min(kblocks, kb0 + kb_half);
                 for (int kb = kb0; kb < kb1; ++kb) {
                     ok = mbar_wait(&full_bar[st], ph, abort_flag);
@@ -250,9 +458,8 @@ __global__ void __launch_bounds__(kHeadThreads, 1) head_proj_kernel(const __grid
         const int lane_base = (warp & 3) * 32;
         bool ok = true;
         int it = 0;
-        for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++it) {
-            const int t2 = tile / kSplit;
-            const int tn = t2 % P.tiles_n, tm = t2 / P.tiles_n;
+        for (int tile = first_tile; tile < total_tiles && ok; tile += tile_step, ++it) {
+            const int tn = tile % P.tiles_n, tm = tile / P.tiles_n;
             const int ab = it & 1;
             const uint32_t acc_ph = (it >> 1) & 1;
             ok = mbar_wait(&acc_full[ab], acc_ph, abort_flag);
@@ -261,7 +468,9 @@ __global__ void __launch_bounds__(kHeadThreads, 1) head_proj_kernel(const __grid
             const int v = P.v_begin + tm * kBM + lane_base + lane;  // this thread's token id
             const bool v_ok = v < P.v_end;
             const uint32_t taddr = tmem_base + (static_cast<uint32_t>(lane_base) << 16) + static_cast<uint32_t>(ab * P.BN);
-            epilogue_store<KSPLIT>(P, taddr, tn, v, v_ok);
+            // each block hands the other the chunks that one will finish; the stores follow once the pair has met
+            (void)tn, (void)v_ok;
+            epilogue_send(P, taddr, lane_base + lane, map_shared_to_cta(smem + P.xchg_off, part ^ 1), part ^ 1);
             tcgen05_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(&acc_empty[ab]);
@@ -274,6 +483,22 @@ __global__ void __launch_bounds__(kHeadThreads, 1) head_proj_kernel(const __grid
 
     tcgen05_fence_before();
     __syncthreads();
+    {
+        // every thread of both blocks gets here, whatever happened above: each block now holds its partner's sums for
+        // the chunks it owns
+        cluster_sync_all();
+        if (warp >= 2 && first_tile < total_tiles && !*abort_flag) {
+            tcgen05_fence_after();
+            const int lane_base = (warp & 3) * 32;
+            const int tn = first_tile % P.tiles_n, tm = first_tile / P.tiles_n;
+            const int v = P.v_begin + tm * kBM + lane_base + lane;
+            const uint32_t taddr = tmem_base + (static_cast<uint32_t>(lane_base) << 16);
+            epilogue_store<true>(P, taddr, tn, v, v < P.v_end, part, 2, reinterpret_cast<const float *>(smem + P.xchg_off),
+                                 lane_base + lane);
+            tcgen05_fence_before();
+        }
+        __syncthreads();
+    }
     if (warp == 1) {
         tcgen05_fence_after();
         tmem_dealloc(tmem_base, kTmemCols);
@@ -466,17 +691,6 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kPairThreads, 1)
 }
 
 
-// Zeroes logits[M][v_begin, v_end) ahead of a call whose tiles are split along the hidden dimension.
-__global__ void head_zero_kernel(float *logits, int M, int V, int v_begin, int n)
-{
-    hawk::allow_dependent_launch();
-    hawk::grid_dependency_wait();
-    const long long idx = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x;
-    if (idx >= static_cast<long long>(M) * n) return;
-    const int m = static_cast<int>(idx / n), c = static_cast<int>(idx - static_cast<long long>(m) * n);
-    logits[static_cast<size_t>(m) * V + v_begin + c] = 0.f;
-}
-
 }  // namespace
 
 hawk_status hawk_host::check_head_proj_args(const void *x, const void *w, const float *logits, int M, int hidden, int V,
@@ -543,7 +757,11 @@ hawk_status head_proj_impl(const void *x, const void *w, float *logits, int M, i
     const int tile_rows = use_pair ? 2 * kBM : kBM;  // token ids per tile
     P.tiles_m = (v_end - v_begin + tile_rows - 1) / tile_rows;
     P.stage_bytes = kATileBytes + x_box_rows * kBK * 2 * (pairs != 0 && !use_pair ? 2 : 1);
-    const int smem_budget = 200 * 1024;
+    // few tiles and a long hidden dimension (a narrow valid range of a wide model): a pair of blocks per tile, each
+    // over half of the hidden dimension, so that twice as many SMs stream the weights
+    P.ksplit = (!use_pair && 2 * P.tiles_m * P.tiles_n <= sm_count && hidden / kBK >= 16) ? 2 : 1;
+    const int xchg_bytes = P.ksplit > 1 ? kBM * P.BN * 4 : 0;  // block 1's sums, received by block 0
+    const int smem_budget = 200 * 1024 - xchg_bytes;
     int stages = smem_budget / P.stage_bytes;
     if (stages > kMaxStages) stages = kMaxStages;
     if (stages < 2) return HAWK_ERR_UNSUPPORTED;
@@ -558,15 +776,16 @@ hawk_status head_proj_impl(const void *x, const void *w, float *logits, int M, i
         return HAWK_ERR_CUDA;
 
     // always ask for enough shared memory that a second block cannot share the SM: each block owns all of TMEM
-    const size_t smem_bytes = 1024 + static_cast<size_t>(stages) * P.stage_bytes + (3 * kMaxStages + 4) * 8 + 64;
+    P.xchg_off = ((stages * P.stage_bytes + (3 * kMaxStages + 4) * 8 + 64 + 1023) / 1024) * 1024;
+    const size_t smem_bytes = 1024 + static_cast<size_t>(P.xchg_off) + xchg_bytes;
     const size_t smem_req = smem_bytes < 120 * 1024 ? 120 * 1024 : smem_bytes;
     int device = 0;
     if (cudaGetDevice(&device) != cudaSuccess || device < 0 || device >= 64) return HAWK_ERR_CUDA;
     static std::atomic<unsigned long long> attr_done{0};  // per device: the dynamic shared memory limit is a per-device attribute
     if (!((attr_done.load(std::memory_order_relaxed) >> device) & 1ull)) {
-        if (cudaFuncSetAttribute(head_proj_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) !=
+        if (cudaFuncSetAttribute(head_proj_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) !=
                 cudaSuccess ||
-            cudaFuncSetAttribute(head_proj_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) !=
+            cudaFuncSetAttribute(head_proj_split_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) !=
                 cudaSuccess ||
             cudaFuncSetAttribute(head_proj_pair_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) !=
                 cudaSuccess ||
@@ -575,19 +794,8 @@ hawk_status head_proj_impl(const void *x, const void *w, float *logits, int M, i
             return HAWK_ERR_CUDA;
         attr_done.fetch_or(1ull << device, std::memory_order_relaxed);
     }
-    // few tiles and a long hidden dimension (a narrow valid range of a wide model): split every tile's k-blocks
-    // over two blocks so that twice as many SMs stream the weights; plain logits only (the guidance combine
-    // of the other form is applied to complete sums)
-    P.ksplit = (!use_pair && pairs == 0 && 2 * P.tiles_m * P.tiles_n <= sm_count && hidden / kBK >= 16) ? 2 : 1;
-    const int total_tiles = P.tiles_m * P.tiles_n * P.ksplit;
+    const int total_tiles = P.tiles_m * P.tiles_n;
     cudaError_t err;
-    if (P.ksplit > 1) {
-        const int n = v_end - v_begin;
-        const long long cells = static_cast<long long>(M) * n;
-        err = hawk_host::launch_dependent(head_zero_kernel, dim3(static_cast<unsigned>((cells + 255) / 256)), dim3(256), 0,
-                                          reinterpret_cast<cudaStream_t>(stream), logits, M, V, v_begin, n);
-        if (err != cudaSuccess) return HAWK_ERR_CUDA;
-    }
     if (use_pair) {
         // pairs that can be resident at once (an SM without a free neighbour in its group takes none): a
         // persistent grid larger than that would run its last pairs after all the others have finished
@@ -611,10 +819,27 @@ hawk_status head_proj_impl(const void *x, const void *w, float *logits, int M, i
                                           dim3(2 * n_pairs), dim3(kPairThreads), smem_req,
                                           reinterpret_cast<cudaStream_t>(stream), map_w, map_x, P);
     } else {
-        const int grid = total_tiles < sm_count ? total_tiles : sm_count;
-        err = hawk_host::launch_dependent(P.ksplit > 1 ? head_proj_kernel<true> : head_proj_kernel<false>, dim3(grid),
-                                          dim3(kHeadThreads), smem_req, reinterpret_cast<cudaStream_t>(stream), map_w,
-                                          map_x, P);
+        if (P.ksplit > 1) {  // one cluster of two blocks per tile
+            cudaLaunchAttribute attr[2];
+            attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+            attr[0].val.programmaticStreamSerializationAllowed = 1;
+            attr[1].id = cudaLaunchAttributeClusterDimension;
+            attr[1].val.clusterDim.x = 2;
+            attr[1].val.clusterDim.y = 1;
+            attr[1].val.clusterDim.z = 1;
+            cudaLaunchConfig_t cfg = {};
+            cfg.gridDim = dim3(2 * total_tiles);
+            cfg.blockDim = dim3(kHeadThreads);
+            cfg.dynamicSmemBytes = smem_req;
+            cfg.stream = reinterpret_cast<cudaStream_t>(stream);
+            cfg.attrs = attr;
+            cfg.numAttrs = 2;
+            err = cudaLaunchKernelEx(&cfg, head_proj_split_kernel, map_w, map_x, P);
+        } else {
+            const int grid = total_tiles < sm_count ? total_tiles : sm_count;
+            err = hawk_host::launch_dependent(head_proj_kernel, dim3(grid), dim3(kHeadThreads), smem_req,
+                                              reinterpret_cast<cudaStream_t>(stream), map_w, map_x, P);
+        }
     }
     return err == cudaSuccess ? HAWK_OK : HAWK_ERR_CUDA;
 }
