@@ -53,9 +53,9 @@ NOMINAL_BF16_TFLOPS = 2250.0   # dense bf16
 # DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) of one hawk_verify_attn call, attention kernel
 # plus merge kernel, from the ncu captures summarised in profiles/ (not measured by this script); an entry is
 # dropped when the attention kernels change and no new capture exists.
-ATTN_TRAFFIC_BYTES = {2: 94_541_000 + 3_350_000,                 # attention kernel read + write (no merge kernel at this shape)
-                      4: 317_136_000 + 3_765_000,               # the same at the 7B shape
-                      5: 679_408_000 + 4_620_000 + 4_757_000}   # attention read + write, merge kernel read
+ATTN_TRAFFIC_BYTES = {2: 94_543_000 + 3_216_000,                 # attention kernel read + write (no merge kernel at this shape)
+                      4: 317_123_000 + 3_759_000,               # the same at the 7B shape
+                      5: 679_410_000 + 4_565_000 + 4_757_000}   # attention read + write, merge kernel read
 
 
 def measured_peaks():
@@ -351,7 +351,7 @@ def accept_traffic_model(cfg, accept_len):
 
 # DRAM bytes of one hawk_cfg_accept call from the ncu captures summarised in profiles/ (rows kernel, read + write;
 # at workload 5 the figure depends on how many rows see an earlier rejection in time: 33 to 38 MB in two launches)
-ACCEPT_TRAFFIC_BYTES = {2: 6_066_000, 4: 1_877_000, 5: 35_575_000}
+ACCEPT_TRAFFIC_BYTES = {2: 6_066_000, 4: 1_877_000, 5: 35_968_000}
 
 
 def launches_per_step(cfg, first, sms):
